@@ -1,0 +1,450 @@
+/*
+ * CPU oracle for layer-wise stochastic quantization and the QODA update.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, single-threaded statement
+ * of what the method computes, written from the paper's equations.  It shares no code,
+ * header, table or constant generator with the CUDA library and must never be linked
+ * into, or called from, the product path.  Only the tests, the smoke check and the
+ * benchmark's CPU-baseline leg may use it.
+ *
+ * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC lq_oracle.c -lm
+ * (no contraction, no fast-math: every fp32 operation below is one IEEE-rounded step).
+ *
+ * Parity status of each part against the paper:
+ *   philox, norm, quantizer, pack, histogram, decode/aggregate, QODA update: pinned by
+ *     the CPU tests (known-answer vectors, closed forms, brute force, invariants).
+ *   level fit (orc_fit_levels): the paper states the objective (Section 3.2, the
+ *     variance minimisation after Eq. MQV and the CDF weights) but no solver, so the
+ *     solver here is this build's own: "parity unpinned" against the paper; it is
+ *     pinned only through properties of the objective (descent, stationarity, the
+ *     uniform-density closed form, brute-force search on small cases).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------------------
+ * Counter-based random numbers: Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw,
+ * "Parallel random numbers: as easy as 1, 2, 3", SC'11).  The paper's quantizer needs one
+ * independent uniform per coordinate (Section 3.1, definition of q_l(u)); keying the
+ * stream on (seed, step, worker, layer, index) is this build's choice so that a CPU and a
+ * GPU draw the same value for the same coordinate.
+ * ---------------------------------------------------------------------------------- */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int round = 0; round < 10; ++round) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Uniform in [0,1) for coordinate `index` of (worker, layer) at iteration `step`:
+ * key = (seed low, seed high), counter = (index / 4, layer, worker, step), the coordinate
+ * takes output word index % 4, and rho = (word >> 8) * 2^-24 (exact in fp32). */
+float orc_uniform(uint64_t seed, uint32_t step, uint32_t worker, uint32_t layer, uint64_t index)
+{
+    uint32_t ctr[4] = { (uint32_t)(index >> 2), layer, worker, step };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return (float)(out[index & 3] >> 8) * 5.9604644775390625e-08f; /* 2^-24 */
+}
+
+/* ------------------------------------------------------------------------------------
+ * L^q norm of one layer (Section 2.2: v is represented by (||v||_q, sign, u)).
+ * q = 0 stands for the infinity norm.  Accumulated in fp64, returned rounded to fp32
+ * (the message carries the norm as a 32-bit float, Section 3.2).
+ * status: 0 ok, 1 zero norm (below the smallest normal float), 2 non-finite.
+ * In both flagged cases the returned norm is 0 and the layer's message is all zero.
+ * ---------------------------------------------------------------------------------- */
+float orc_layer_norm(const float* v, int64_t d, int q, int* status)
+{
+    double acc = 0.0;
+    int bad = 0;
+    for (int64_t i = 0; i < d; ++i) {
+        double a = fabs((double)v[i]);
+        if (!(a <= 3.4028234663852886e38)) bad = 1;      /* NaN or infinity */
+        if (q == 0)      { if (a > acc) acc = a; }
+        else if (q == 1) acc += a;
+        else if (q == 2) acc += a * a;
+        else { double p = a; for (int r = 1; r < q; ++r) p *= a; acc += p; }
+    }
+    double n64;
+    if (q == 0 || q == 1) n64 = acc;
+    else if (q == 2)      n64 = sqrt(acc);
+    else                  n64 = pow(acc, 1.0 / (double)q);
+    float n = (float)n64;
+    int st = 0;
+    if (bad || !(n64 == n64) || isinf(n64) || isinf(n)) st = 2;
+    else if (n < 1.17549435e-38f) st = 1;
+    if (status) *status = st;
+    return st ? 0.0f : n;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Stochastic quantization of one layer (Section 3.1).  For each coordinate:
+ *   u   = min(|v| * (1/N), 1)                       normalised magnitude (Section 2.2)
+ *   tau = the largest j <= n-2 with level[j] <= u   (so u = 1 falls in the last interval)
+ *   up with probability xi(u) = (u - l_tau) / (l_{tau+1} - l_tau), decided as
+ *        rho * (l_{tau+1} - l_tau) < (u - l_tau)     with rho the coordinate's uniform
+ *   idx = tau + up,  sign = sign bit of v.
+ * `near` counts coordinates whose decision is within 1e-6 (relative to the interval)
+ * of the threshold.  norm == 0 gives an all-zero message.
+ * ---------------------------------------------------------------------------------- */
+void orc_quantize_layer(const float* v, int64_t d, float norm, const float* level, int n,
+                        uint64_t seed, uint32_t step, uint32_t worker, uint32_t layer,
+                        uint8_t* idx, uint8_t* sign, int64_t* near)
+{
+    int64_t near_count = 0;
+    if (!(norm > 0.0f)) {
+        memset(idx, 0, (size_t)d); memset(sign, 0, (size_t)d);
+        if (near) *near = 0;
+        return;
+    }
+    const float r = 1.0f / norm;
+    for (int64_t i = 0; i < d; ++i) {
+        float a = fabsf(v[i]);
+        float u = a * r;
+        if (u > 1.0f) u = 1.0f;
+        int tau = 0;
+        for (int j = 1; j <= n - 2; ++j) if (level[j] <= u) tau = j;
+        float num = u - level[tau];
+        float den = level[tau + 1] - level[tau];
+        float rho = orc_uniform(seed, step, worker, layer, (uint64_t)i);
+        float t = rho * den;
+        int up = (t < num) ? 1 : 0;
+        if (fabsf(t - num) <= 1e-6f * den) ++near_count;
+        idx[i] = (uint8_t)(tau + up);
+        sign[i] = (uint8_t)(signbit(v[i]) ? 1 : 0);
+    }
+    if (near) *near = near_count;
+}
+
+/* Probability of rounding up for one normalised value (xi(u), Section 3.1), in fp64. */
+double orc_round_up_probability(double u, const float* level, int n, int* tau_out)
+{
+    int tau = 0;
+    for (int j = 1; j <= n - 2; ++j) if ((double)level[j] <= u) tau = j;
+    if (tau_out) *tau_out = tau;
+    return (u - (double)level[tau]) / ((double)level[tau + 1] - (double)level[tau]);
+}
+
+/* ------------------------------------------------------------------------------------
+ * Fixed-width message layout (Section 3.2: a 32-bit float norm, one sign bit and one
+ * integer code per coordinate; Section 7.1 footnote: no entropy code on top).
+ * The physical layout is this build's:
+ *   a layer of d coordinates with b-bit codes is cut into blocks of 1024 coordinates
+ *   (the last one zero-padded); a block is (b+1) planes of 32 words; coordinate c of a
+ *   block belongs to lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane;
+ *   plane 0 holds the signs (bit p of the lane's word); planes 1..b hold, per lane, the
+ *   32 codes as one little-endian string of 32*b bits with code p at bit offset p*b.
+ * ---------------------------------------------------------------------------------- */
+int64_t orc_packed_words(int64_t d, int b)
+{
+    return ((d + 1023) / 1024) * 32 * (int64_t)(b + 1);
+}
+
+static void locate(int64_t i, int b, int64_t* block_base, int* lane, int* p)
+{
+    int64_t blk = i / 1024;
+    int c = (int)(i % 1024);
+    *block_base = blk * 32 * (int64_t)(b + 1);
+    *lane = (c / 4) % 32;
+    *p = 4 * (c / 128) + c % 4;
+}
+
+void orc_pack_layer(const uint8_t* idx, const uint8_t* sign, int64_t d, int b, uint32_t* words)
+{
+    memset(words, 0, (size_t)orc_packed_words(d, b) * sizeof(uint32_t));
+    for (int64_t i = 0; i < d; ++i) {
+        int64_t base; int lane, p;
+        locate(i, b, &base, &lane, &p);
+        if (sign[i]) words[base + lane] |= (uint32_t)1 << p;
+        for (int bit = 0; bit < b; ++bit) {
+            if ((idx[i] >> bit) & 1) {
+                int pos = p * b + bit;               /* position in the 32*b-bit string */
+                words[base + (int64_t)(1 + pos / 32) * 32 + lane] |= (uint32_t)1 << (pos % 32);
+            }
+        }
+    }
+}
+
+void orc_unpack_layer(const uint32_t* words, int64_t d, int b, uint8_t* idx, uint8_t* sign)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        int64_t base; int lane, p;
+        locate(i, b, &base, &lane, &p);
+        sign[i] = (uint8_t)((words[base + lane] >> p) & 1u);
+        unsigned code = 0;
+        for (int bit = 0; bit < b; ++bit) {
+            int pos = p * b + bit;
+            code |= ((words[base + (int64_t)(1 + pos / 32) * 32 + lane] >> (pos % 32)) & 1u) << bit;
+        }
+        idx[i] = (uint8_t)code;
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Histogram of normalised magnitudes of one layer (Algorithm 1, line 4: estimate the
+ * distribution of normalised dual vectors).  The binning is this build's: 386 bins,
+ * bin 0 = [0, 2^-24), then 16 bins per octave with edges 2^e * (1 + m/16) up to 1,
+ * and the last bin holds u = 1 only.  The bin is found here by comparing against the
+ * edges, one by one.
+ * ---------------------------------------------------------------------------------- */
+#define ORC_NUM_BINS 386
+
+double orc_bin_edge(int i)      /* lower edge of bin i, i = 0..386 (edge 385 = 1) */
+{
+    if (i <= 0) return 0.0;
+    if (i > 385) return 1.0 + 1.0 / 16.0;
+    int o = (i - 1) / 16, m = (i - 1) % 16;
+    return ldexp(1.0 + (double)m / 16.0, -24 + o);
+}
+
+void orc_histogram_layer(const float* v, int64_t d, float norm, uint32_t* hist)
+{
+    if (!(norm > 0.0f)) return;
+    double edge[ORC_NUM_BINS + 1];
+    for (int i = 0; i <= ORC_NUM_BINS; ++i) edge[i] = orc_bin_edge(i);
+    const float r = 1.0f / norm;
+    for (int64_t i = 0; i < d; ++i) {
+        float u = fabsf(v[i]) * r;
+        if (u > 1.0f) u = 1.0f;
+        int bin = 0;
+        while (bin < ORC_NUM_BINS - 1 && (double)u >= edge[bin + 1]) ++bin;
+        hist[bin] += 1u;
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * Level fit (Section 3.2: minimise sum_j int_{l_j}^{l_{j+1}} sigma_Q^2(u; l) dF~(u), with
+ * F~ the sum of the Z sampled vectors' CDFs weighted by lambda_z = N_z^2 / sum N_z^2).
+ * The paper names no solver; this one is the build's own ("parity unpinned"):
+ *   F~ is taken piecewise linear from the merged histogram (uniform density in a bin);
+ *   the mass at u = 1 (last bin) never contributes variance and is left out;
+ *   start: quantiles j/(n-1) of the mass above bin 0;
+ *   sweeps: exact coordinate minimisation of one interior level given its neighbours
+ *     a < c, i.e. F~(l) = F~(c) - int_a^c (u-a)/(c-a) dF~(u)  (the first-order condition
+ *     int_a^l (u-a) dF~ = int_l^c (c-u) dF~), odd levels first, then even levels;
+ *   up to 100 sweeps, stopping when no level moved by more than 1e-13 relative;
+ *   round to fp32 and force strict monotonicity by single-ulp steps.
+ * Returns 1 if levels were written, 0 if there was no usable mass (levels untouched).
+ * hist is [Z][stride] counts, norms are the Z vectors' fp32 norms, d the layer size.
+ * ---------------------------------------------------------------------------------- */
+typedef struct {
+    double e[ORC_NUM_BINS + 1];       /* bin edges, e[385] = 1 */
+    double mass[ORC_NUM_BINS];        /* weighted mass of bins 0..384 (bin 385 unused) */
+    double F[ORC_NUM_BINS + 1];       /* cumulative mass at the edges */
+    double M1[ORC_NUM_BINS + 1];      /* cumulative first moment at the edges */
+} orc_density;
+
+static int find_bin(const orc_density* D, double x)
+{
+    int lo = 0, hi = 384;             /* largest i in [0,384] with e[i] <= x */
+    while (lo < hi) {
+        int mid = (lo + hi + 1) / 2;
+        if (D->e[mid] <= x) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+static double cdf_at(const orc_density* D, double x, double* first_moment)
+{
+    int i = find_bin(D, x);
+    double theta = (x - D->e[i]) / (D->e[i + 1] - D->e[i]);
+    if (theta > 1.0) theta = 1.0;
+    double part = D->mass[i] * theta;
+    if (first_moment) *first_moment = D->M1[i] + part * ((D->e[i] + x) * 0.5);
+    return D->F[i] + part;
+}
+
+static double cdf_inverse(const orc_density* D, double y)
+{
+    int lo = 0, hi = 385;             /* smallest i in [0,385] with F[i+1] > y; 385 = none */
+    while (lo < hi) {
+        int mid = (lo + hi) / 2;
+        if (D->F[mid + 1] > y) hi = mid; else lo = mid + 1;
+    }
+    if (lo >= 385) return 1.0;
+    double t = (y - D->F[lo]) / D->mass[lo];
+    if (t < 0.0) t = 0.0;
+    return D->e[lo] + t * (D->e[lo + 1] - D->e[lo]);
+}
+
+int orc_fit_levels(const uint32_t* hist, int64_t stride, const float* norms, int Z,
+                   int64_t d, int n, float* level_out)
+{
+    static orc_density D;             /* single-threaded oracle: static storage is fine */
+    if (n < 3 || d <= 0) return 0;
+    double wsum = 0.0;
+    for (int z = 0; z < Z; ++z) wsum += (double)norms[z] * (double)norms[z];
+    if (!(wsum > 0.0)) return 0;
+    for (int i = 0; i <= 385; ++i) D.e[i] = orc_bin_edge(i);
+    for (int i = 0; i < 385; ++i) {
+        double m = 0.0;
+        for (int z = 0; z < Z; ++z) {
+            double lambda = ((double)norms[z] * (double)norms[z]) / wsum;
+            m += lambda * (double)hist[(int64_t)z * stride + i];
+        }
+        D.mass[i] = m / (double)d;
+    }
+    D.F[0] = 0.0; D.M1[0] = 0.0;
+    for (int i = 0; i < 385; ++i) {
+        D.F[i + 1] = D.F[i] + D.mass[i];
+        D.M1[i + 1] = D.M1[i] + D.mass[i] * ((D.e[i] + D.e[i + 1]) * 0.5);
+    }
+    double total = D.F[385], above = total - D.mass[0];
+    if (!(above > 0.0)) return 0;
+
+    double l[256];
+    l[0] = 0.0; l[n - 1] = 1.0;
+    for (int j = 1; j <= n - 2; ++j)
+        l[j] = cdf_inverse(&D, D.mass[0] + above * ((double)j / (double)(n - 1)));
+
+    for (int sweep = 0; sweep < 100; ++sweep) {
+        double moved = 0.0;
+        for (int parity = 1; parity >= 0; --parity) {
+            for (int j = 1; j <= n - 2; ++j) {
+                if ((j & 1) != parity) continue;
+                double a = l[j - 1], c = l[j + 1], b;
+                if (!(c > a)) continue;
+                double m1a, m1c;
+                double Fa = cdf_at(&D, a, &m1a), Fc = cdf_at(&D, c, &m1c);
+                double mass_ac = Fc - Fa;
+                if (!(mass_ac > 0.0)) b = (a + c) * 0.5;
+                else {
+                    double target = Fc - ((m1c - m1a) - a * mass_ac) / (c - a);
+                    b = cdf_inverse(&D, target);
+                    if (b < a) b = a;
+                    if (b > c) b = c;
+                }
+                double rel = fabs(b - l[j]) / (fabs(b) > 1e-300 ? fabs(b) : 1e-300);
+                if (rel > moved) moved = rel;
+                l[j] = b;
+            }
+        }
+        if (moved <= 1e-13) break;
+    }
+
+    level_out[0] = 0.0f; level_out[n - 1] = 1.0f;
+    for (int j = 1; j <= n - 2; ++j) {
+        float f = (float)l[j];
+        float floor_ = nextafterf(level_out[j - 1], 2.0f);
+        level_out[j] = f > floor_ ? f : floor_;
+    }
+    for (int j = n - 2; j >= 1; --j) {
+        float ceil_ = nextafterf(level_out[j + 1], -1.0f);
+        if (level_out[j] > ceil_) level_out[j] = ceil_;
+    }
+    return 1;
+}
+
+/* Objective of the fit evaluated from the same piecewise-uniform density (used by the
+ * tests to check descent against levels that did not come from the solver). */
+double orc_fit_objective(const uint32_t* hist, int64_t stride, const float* norms, int Z,
+                         int64_t d, const float* level, int n)
+{
+    double wsum = 0.0, total = 0.0;
+    for (int z = 0; z < Z; ++z) wsum += (double)norms[z] * (double)norms[z];
+    if (!(wsum > 0.0)) return 0.0;
+    for (int i = 0; i < 385; ++i) {
+        double m = 0.0;
+        for (int z = 0; z < Z; ++z)
+            m += (((double)norms[z] * (double)norms[z]) / wsum) * (double)hist[(int64_t)z * stride + i];
+        m /= (double)d;
+        if (m == 0.0) continue;
+        double lo = orc_bin_edge(i), hi = orc_bin_edge(i + 1), dens = m / (hi - lo);
+        /* cut the bin at every level that falls inside it and integrate
+         * (l_{j+1} - u)(u - l_j) exactly on each piece */
+        double x0 = lo;
+        while (x0 < hi) {
+            int j = 0;
+            for (int t = 1; t <= n - 2; ++t) if ((double)level[t] <= x0) j = t;
+            double a = level[j], c = level[j + 1];
+            double x1 = c < hi ? c : hi;
+            if (!(x1 > x0)) break;
+            /* int (c-u)(u-a) du = [-(u^3)/3 + (a+c)u^2/2 - a c u] */
+            double P0 = -x0 * x0 * x0 / 3.0 + (a + c) * x0 * x0 * 0.5 - a * c * x0;
+            double P1 = -x1 * x1 * x1 / 3.0 + (a + c) * x1 * x1 * 0.5 - a * c * x1;
+            total += dens * (P1 - P0);
+            x0 = x1;
+        }
+    }
+    return total;
+}
+
+/* ------------------------------------------------------------------------------------
+ * DECODE of one layer (Section 3.2; Algorithm 1 line 15): V^_i = N * sign_i * l_{idx_i},
+ * evaluated as one fp32 multiply N * l_idx with the sign applied afterwards.
+ * ---------------------------------------------------------------------------------- */
+void orc_decode_layer(const uint8_t* idx, const uint8_t* sign, int64_t d, float norm,
+                      const float* level, float* out)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        float mag = norm * level[idx[i]];
+        out[i] = sign[i] ? -mag : mag;
+    }
+}
+
+/* Mean of K decoded vectors, accumulated in fp32 in worker order, then scaled by the
+ * fp32 reciprocal of K (Algorithm 1 lines 10 and 17: sum_k V^_k / K).
+ * decoded is [K][d]. */
+void orc_aggregate(const float* decoded, int K, int64_t d, float* gbar)
+{
+    const float invK = 1.0f / (float)K;
+    for (int64_t i = 0; i < d; ++i) {
+        float acc = 0.0f;
+        for (int k = 0; k < K; ++k) acc = acc + decoded[(int64_t)k * d + i];
+        gbar[i] = acc * invK;
+    }
+}
+
+/* sum_i (cur_i - prev_i)^2 in fp64 with exact differences: one worker-layer term of the
+ * adaptive step size (Eq. general_stepsize: ||V^_{k,s+1/2} - V^_{k,s-1/2}||^2). */
+double orc_sq_diff(const float* cur, const float* prev, int64_t d)
+{
+    double acc = 0.0;
+    for (int64_t i = 0; i < d; ++i) {
+        double t = (double)cur[i] - (prev ? (double)prev[i] : 0.0);
+        acc += t * t;
+    }
+    return acc;
+}
+
+/* eta_{t+1} = gamma_{t+1} = (1 + S_t)^(-1/2), S_t = S_{t-1} + sum_k ||.||^2 / K^2
+ * (Eq. general_stepsize).  Returns the new S; *eta receives the fp32 step size. */
+double orc_step_size(double S_prev, double sum_sq_diff, int K, float* eta)
+{
+    double S = S_prev + sum_sq_diff / ((double)K * (double)K);
+    *eta = (float)(1.0 / sqrt(1.0 + S));
+    return S;
+}
+
+/* Optimistic dual averaging update (Eq. ODA; Algorithm 1 lines 17, 18 and, for the next
+ * iteration, line 10), each written as one fp32 operation:
+ *   Y_{t+1}   = Y_t - gbar
+ *   X_{t+1}   = fma(eta, Y_{t+1}, X_1)
+ *   X_{t+3/2} = fma(-eta, gbar, X_{t+1})        (gamma_{t+1} = eta_{t+1})
+ * X may be NULL. */
+void orc_qoda_update(const float* gbar, const float* X1, float* Y, float* Xhalf, float* X,
+                     float eta, int64_t d)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        float y = Y[i] - gbar[i];
+        float x = fmaf(eta, y, X1[i]);
+        Y[i] = y;
+        if (X) X[i] = x;
+        Xhalf[i] = fmaf(-eta, gbar[i], x);
+    }
+}

@@ -1,0 +1,203 @@
+"""Pins of the CPU oracle's level fit and of its QODA loop (no CUDA involved).
+
+The paper gives the fit's objective but no solver, so the solver is pinned only through
+properties of that objective; the QODA update is pinned through the identities of the
+paper's appendix and through its behaviour on bilinear games.
+"""
+import math
+
+import numpy as np
+import pytest
+
+SEED = 0x5EED0DA
+
+
+def _hist_of(orc, u):
+    """Histogram of given normalised magnitudes (norm 1 under the max norm)."""
+    v = np.asarray(u, np.float32)
+    v = np.concatenate([v, np.float32([1.0])])              # makes the max norm exactly 1
+    h = orc.histogram_layer(v, 1.0)
+    h[385] -= 1
+    return h
+
+
+def _sample_objective(u, levels):
+    """(1/d) sum_i (l_{tau+1}-u_i)(u_i-l_tau): Eq. (Var) per unit squared norm, from the samples."""
+    lv = np.asarray(levels, np.float64)
+    tau = np.clip(np.searchsorted(lv, u, side="right") - 1, 0, len(lv) - 2)
+    return float(np.mean((lv[tau + 1] - u) * (u - lv[tau])))
+
+
+def test_uniform_density_gives_uniform_levels(orc):
+    """For a uniform density on [0,1] the stationarity condition reads (b-a)^2 = (c-b)^2,
+    so the minimiser is the uniform grid j/(n-1)."""
+    N = 1 << 21
+    u = (np.arange(N) + 0.5) / N
+    h = _hist_of(orc, u)
+    for n in (4, 8, 16):
+        lv = orc.fit_levels(h[None, :], [1.0], N, n)
+        assert np.allclose(lv, np.arange(n) / (n - 1), atol=2e-4)
+
+
+@pytest.mark.parametrize("dist", ["halfnormal", "laplace", "student"])
+def test_fit_is_a_minimum_of_the_objective(orc, dist):
+    rng = np.random.default_rng(42)
+    d = 60000
+    x = {"halfnormal": rng.standard_normal(d), "laplace": rng.laplace(size=d),
+         "student": rng.standard_t(3, size=d)}[dist].astype(np.float32)
+    norm, _ = orc.layer_norm(x, 2)
+    u = np.minimum(np.abs(x) * (np.float32(1) / norm), np.float32(1)).astype(np.float64)
+    h = orc.histogram_layer(x, norm)
+    n = 16
+    lv = orc.fit_levels(h[None, :], [norm], d, n)
+    assert lv[0] == 0 and lv[-1] == 1 and np.all(np.diff(lv) > 0)
+    f_fit = orc.fit_objective(h[None, :], [norm], d, lv)
+    # the closed-form objective on the histogram density agrees with the sample sum of Eq. (Var)
+    assert abs(f_fit - _sample_objective(u, lv)) < 0.02 * f_fit
+    # better than uniform levels and than exponential levels 2^-(n-1-j)
+    uni = orc.uniform_levels(4)
+    expo = np.concatenate([[0], 2.0 ** -np.arange(n - 2, -1, -1)]).astype(np.float32)
+    assert f_fit < orc.fit_objective(h[None, :], [norm], d, uni)
+    assert f_fit < orc.fit_objective(h[None, :], [norm], d, expo)
+    # local minimum: random feasible perturbations never improve it (beyond rounding)
+    for _ in range(200):
+        p = lv.astype(np.float64).copy()
+        j = rng.integers(1, n - 1)
+        p[j] += rng.uniform(-0.3, 0.3) * min(p[j] - p[j - 1], p[j + 1] - p[j])
+        assert orc.fit_objective(h[None, :], [norm], d, p.astype(np.float32)) >= f_fit * (1 - 1e-6)
+    # an independent optimiser on the sample objective cannot do noticeably better
+    from scipy.optimize import minimize
+
+    def obj(z):
+        inner = np.sort(1.0 / (1.0 + np.exp(-z)))
+        return _sample_objective(u, np.concatenate([[0.0], inner, [1.0]])) * 1e6
+    z0 = np.log(lv[1:-1].astype(np.float64) / (1 - lv[1:-1].astype(np.float64)))
+    best = minimize(obj, z0 + rng.normal(0, 0.2, n - 2), method="Powell",
+                    options=dict(maxiter=1500, xtol=1e-5, ftol=1e-8)).fun / 1e6
+    # (the fit sees the samples only through 16 bins per octave, which costs a few per cent
+    # in the sparse tail of heavy-tailed data)
+    assert _sample_objective(u, lv) <= best * 1.08
+
+
+def test_stationarity_condition(orc):
+    """At the fitted levels int_a^b (u-a) dF = int_b^c (c-u) dF for every interior level,
+    evaluated directly on the samples."""
+    rng = np.random.default_rng(7)
+    d = 400000
+    x = rng.laplace(size=d).astype(np.float32)
+    norm, _ = orc.layer_norm(x, 2)
+    u = np.abs(x.astype(np.float64)) / float(norm)
+    h = orc.histogram_layer(x, norm)
+    lv = orc.fit_levels(h[None, :], [norm], d, 8).astype(np.float64)
+    for j in range(1, 7):
+        a, b, c = lv[j - 1], lv[j], lv[j + 1]
+        lo, hi = (u >= a) & (u < b), (u >= b) & (u < c)
+        if min(lo.sum(), hi.sum()) < 1000:        # too few samples for a meaningful comparison
+            continue
+        left, right = np.sum((u - a)[lo]), np.sum((c - u)[hi])
+        assert abs(left - right) < 0.01 * max(left, right)
+
+
+def test_layerwise_fit_beats_shared_fit(orc):
+    """Remark after Eq. (MQV): per-layer sequences never lose to one shared sequence."""
+    rng = np.random.default_rng(3)
+    d = 100000
+    xa = rng.standard_normal(d).astype(np.float32)
+    xb = (rng.standard_t(3, size=d) * 0.01).astype(np.float32)
+    na, _ = orc.layer_norm(xa, 2); nb, _ = orc.layer_norm(xb, 2)
+    ha = orc.histogram_layer(xa, na); hb = orc.histogram_layer(xb, nb)
+    la = orc.fit_levels(ha[None], [na], d, 8); lb = orc.fit_levels(hb[None], [nb], d, 8)
+    # shared sequence: fitted on both samples as one type (weights = squared norms)
+    shared = orc.fit_levels(np.stack([ha, hb]), [na, nb], d, 8)
+    wa, wb = float(na) ** 2, float(nb) ** 2
+
+    def total(l1, l2):
+        return wa * orc.fit_objective(ha[None], [na], d, l1) + wb * orc.fit_objective(hb[None], [nb], d, l2)
+    assert total(la, lb) <= total(shared, shared) * (1 + 1e-9)
+
+
+def test_fit_weights_follow_squared_norms(orc):
+    rng = np.random.default_rng(5)
+    d = 50000
+    xa = rng.standard_normal(d).astype(np.float32); xb = rng.laplace(size=d).astype(np.float32)
+    na, _ = orc.layer_norm(xa, 2); nb, _ = orc.layer_norm(xb, 2)
+    ha = orc.histogram_layer(xa, na); hb = orc.histogram_layer(xb, nb)
+    only_a = orc.fit_levels(ha[None], [na], d, 8)
+    both = orc.fit_levels(np.stack([ha, hb]), [na, 0.0], d, 8)       # lambda_b = 0
+    assert np.array_equal(only_a, both)
+    heavy = orc.fit_levels(np.stack([ha, hb]), [na * 1000, nb], d, 8)  # lambda_b = 1e-6
+    assert np.allclose(heavy, only_a, rtol=1e-3)
+    assert orc.fit_levels(np.stack([ha, hb]), [0.0, 0.0], d, 8) is None
+
+
+# ---------------------------------------------------------------------------------- QODA
+def _bilinear_operator(A, z):
+    n = A.shape[0]
+    x, y = z[:n].astype(np.float64), z[n:].astype(np.float64)
+    return np.concatenate([A @ y, -(A.T @ x)])
+
+
+def test_optimism_converges_where_dual_averaging_does_not(orc):
+    """min_x max_y xy, exact operator, K = 1, no quantization: the extrapolated (optimistic)
+    iterates approach the saddle point, plain dual averaging with the same step rule does not."""
+    A = np.array([[1.0]])
+    X1 = np.array([1.0, 1.0], np.float32)
+    Y = np.zeros(2, np.float32); Xh = X1.copy(); X = X1.copy()
+    S, eta = 0.0, np.float32(1.0)
+    prev = None
+    for t in range(3000):
+        V = _bilinear_operator(A, Xh).astype(np.float32)
+        S, eta = orc.step_size(S, orc.sq_diff(V, prev), 1)
+        orc.qoda_update(V, X1, Y, Xh, X, eta)
+        prev = V
+    assert np.linalg.norm(X) < 0.05 * np.linalg.norm(X1)
+    # plain dual averaging: query at X_t itself
+    Yd = np.zeros(2); Xd = X1.astype(np.float64); Sd = 0.0; prevd = np.zeros(2)
+    for t in range(3000):
+        V = _bilinear_operator(A, Xd)
+        Sd += np.sum((V - prevd) ** 2); prevd = V
+        Yd -= V
+        Xd = X1 + Yd / math.sqrt(1 + Sd)
+    assert np.linalg.norm(Xd) > 0.5 * np.linalg.norm(X1)
+
+
+def test_step_size_formula(orc):
+    # eta_{t+1} = (1 + sum_s sum_k ||.||^2 / K^2)^(-1/2), accumulated over calls
+    S, eta = orc.step_size(0.0, 8.0, 2)
+    assert S == 2.0 and eta == np.float32(1 / math.sqrt(3.0))
+    S, eta = orc.step_size(S, 4.0, 2)
+    assert S == 3.0 and eta == np.float32(0.5)
+    a = np.float32([1.0, 2.0, -3.0]); b = np.float32([0.5, 2.0, 1.0])
+    assert orc.sq_diff(a, b) == 0.25 + 16.0 and orc.sq_diff(a, None) == 14.0
+
+
+def test_qoda_identities_with_quantization(orc):
+    """Appendix identity X_t = X_1 - (eta_t / K) sum_{s<t} sum_k V^_{k,s+1/2}, eta non-increasing,
+    X_{t+1/2} = X_t - gamma_t * mean_k V^_{k,t-1/2}; and the gap of the ergodic average decreases
+    on a noisy bilinear game (Theorem 5.5)."""
+    rng = np.random.default_rng(0)
+    n = 32; D = 2 * n; K = 4
+    A = rng.standard_normal((n, n)) / math.sqrt(n)
+    sizes = [16] * 4
+    model = orc.OracleModel(sizes, [4] * 4, 2, K, SEED)
+    X1 = (rng.standard_normal(D) / math.sqrt(D)).astype(np.float32)
+    model.qoda_init(X1)
+    total = np.zeros(D); avg = np.zeros(D); etas = []; gaps = {}
+    R = float(np.linalg.norm(X1))
+    for t in range(1, 1501):
+        Xh = model.Xhalf.copy()
+        avg += Xh
+        F = _bilinear_operator(A, Xh)
+        V = (F[None, :] + 0.1 * rng.standard_normal((K, D))).astype(np.float32)
+        out = model.quantize(V, t)
+        X_before = model.X.copy(); eta_before = model.eta
+        gbar = model.qoda_step()
+        total += out["decoded"].astype(np.float64).sum(axis=0)
+        etas.append(float(model.eta))
+        assert np.allclose(model.X, X1 - float(model.eta) / K * total, rtol=0, atol=2e-5)
+        assert np.allclose(model.Xhalf, model.X.astype(np.float64) - float(model.eta) * gbar, atol=1e-6)
+        if t in (10, 100, 1500):
+            zbar = avg / t
+            gaps[t] = R * np.linalg.norm(_bilinear_operator(A, zbar))
+    assert all(0 < b <= a <= 1 for a, b in zip(etas, etas[1:]))
+    assert gaps[1500] < 0.5 * gaps[100] < 0.5 * gaps[10]
