@@ -1,0 +1,156 @@
+/*
+ * liblq: layer-wise unbiased stochastic quantization and the Quantized Optimistic Dual
+ * Averaging (QODA) update for K data-parallel workers simulated on one GPU.
+ *
+ * Conventions
+ *  - Every function returns an int: LQ_OK (0) or a negative LQ_E* code.  Nothing throws,
+ *    aborts or traps.  lq_last_error() gives a human-readable reason for the calling
+ *    thread's last failure.
+ *  - "dev" pointers are device memory OWNED BY THE CALLER (allocated however the caller
+ *    likes); "host" pointers are ordinary host memory.  The plan owns only its own
+ *    tables and scratch, released by lq_plan_destroy.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that
+ *    take a stream only enqueue work on it and return; they do not synchronise unless
+ *    stated.  Calls on one plan must be issued in stream order by the caller.
+ *  - Argument errors are reported synchronously.  Data problems (NaN/Inf input, zero
+ *    norm) never fault: they set per-(worker, layer) status flags, see lq_get_status.
+ *
+ * Data layout
+ *  - A plan is a ragged list of L layers with sizes d_m, code widths b_m (n_m = 2^b_m levels
+ *    per layer, including 0 and 1), one norm order q, K workers and a 64-bit seed.
+ *  - Gradient-like buffers (grads, X1, Y, Xhalf, X, gbar) are fp32 rows of D_pad =
+ *    lq_plan_padded_elems() elements; layer m starts at element elem_off_m (a multiple of 32)
+ *    and its d_m values are contiguous.  grads is [K][D_pad], row-major.  Elements between
+ *    layers are padding: never interpreted on input, may be overwritten on output.
+ *  - A worker's message is W = lq_plan_packed_words() 32-bit words; packed is [K][W].
+ *    Layer m starts at word_off_m and is cut into blocks of 1024 coordinates (the last one
+ *    zero-padded).  A block is (b+1) planes of 32 words.  Coordinate c of a block belongs to
+ *    lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane.  Plane 0 holds the sign
+ *    bits (bit p of word `lane`); planes 1..b hold, per lane, the 32 level indices as one
+ *    little-endian string of 32*b bits with index p at bit offset p*b (word `plane*32+lane`).
+ *    The norms travel separately as fp32: norms is [K][L].
+ *    (Section 3.2 of the paper fixes the content of a message: a 32-bit float norm, one sign
+ *    bit and one integer code per coordinate; the physical arrangement is this library's.)
+ */
+#ifndef LQ_H_
+#define LQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LQ_OK       0
+#define LQ_EINVAL  (-1)   /* bad argument (NULL, size, range, non-increasing levels, ...) */
+#define LQ_ENOMEM  (-2)   /* host or device allocation failed */
+#define LQ_ECUDA   (-3)   /* a CUDA runtime call failed; see lq_last_error() */
+#define LQ_ESTATE  (-4)   /* call out of order (e.g. qoda_step before qoda_init) */
+
+#define LQ_NUM_BINS     386   /* histogram bins per (worker, layer) */
+#define LQ_HIST_STRIDE  512   /* words between consecutive histograms */
+#define LQ_MAX_BITS     8
+#define LQ_MAX_WORKERS  1024
+
+#define LQ_STATUS_ZERO_NORM  1u  /* layer norm below the smallest normal float: message is all zero */
+#define LQ_STATUS_NONFINITE  2u  /* NaN/Inf in the layer (or norm overflow): message is all zero, norm 0 */
+
+typedef struct lq_plan lq_plan;
+
+/* Plan over a ragged list of layers (Section 3.1: each layer follows its own sequence of
+ * levels; Section 2.2: L^q normalisation).
+ *   layer_sizes [num_layers] host, each in [0, 2^31);  bits [num_layers] host, each in [1, 8];
+ *   q >= 1 is the norm order (1..16), q = 0 selects the infinity norm;
+ *   num_workers in [1, LQ_MAX_WORKERS];  seed keys the Philox4x32-10 stream together with
+ *   (step, worker, layer, coordinate).
+ * Every layer starts with uniform levels j/(2^b-1).  Allocates device tables and scratch on
+ * the current device; may synchronise.  On failure *out is NULL. */
+int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes,
+                   const int32_t* bits, int32_t q, int32_t num_workers, uint64_t seed);
+int lq_plan_destroy(lq_plan* plan);             /* synchronises the device; NULL is accepted */
+
+int64_t lq_plan_padded_elems(const lq_plan* plan);   /* D_pad, or LQ_EINVAL */
+int64_t lq_plan_packed_words(const lq_plan* plan);   /* W, or LQ_EINVAL */
+/* Any of the three outputs may be NULL. */
+int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, int64_t* word_off,
+                       int32_t* num_levels);
+
+/* Level sequence of one layer (Section 3.1: 0 = l_0 < l_1 < ... < l_{n-1} = 1, n = 2^b).
+ * host_levels [n] host.  set: validates (n must equal 2^b, strictly increasing, ends 0 and 1)
+ * and stages the sequence; it is used from the next lq_quantize_pack on.  get: returns the
+ * staged sequence (the most recent of set / fit).  Both synchronise the device. */
+int lq_set_levels(lq_plan* plan, int32_t layer, const float* host_levels, int32_t n);
+int lq_get_levels(const lq_plan* plan, int32_t layer, float* host_levels, int32_t n);
+
+/* Per-layer L^q norms only (Section 2.2): norms[k][m] = fp32(||grads[k][layer m]||_q),
+ * accumulated in fp64.  grads dev [K][D_pad]; norms dev [K][L].  Updates the status flags. */
+int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream);
+
+/* ENCODE for all K workers (Algorithm 1 line 12; Section 3.1 quantizer, Section 3.2 message):
+ * per-layer norm, normalisation u = min(|v| * (1/N), 1), stochastic rounding of u between its
+ * two neighbouring levels (up with probability (u - l_tau)/(l_{tau+1} - l_tau), uniforms from
+ * Philox keyed (seed, step, worker, layer, coordinate)), sign and index packing.
+ *   grads dev [K][D_pad];  packed dev [K][W] (fully overwritten);  norms dev [K][L] out;
+ *   hist: NULL, or dev [K][L][LQ_HIST_STRIDE] u32 histograms of u, ADDED to (caller zeroes
+ *     them); bin 0 = [0,2^-24), then 16 bins per octave up to 1, bin 385 = {1}
+ *     (Algorithm 1 line 4);
+ *   prev_packed / prev_norms: the message this plan produced in its previous
+ *     lq_quantize_pack call (dev [K][W], [K][L]), or both NULL when there is none
+ *     (V^_{k,1/2} = 0).  Used for the step-size statistic
+ *     sum_k ||V^_{k,t+1/2} - V^_{k,t-1/2}||^2 of Eq. (general_stepsize), which is left
+ *     inside the plan for the next qoda_step.  The previous message is decoded with the
+ *     levels it was encoded with, even if the levels were changed in between.
+ *   prev_packed must not alias packed. */
+int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t* packed,
+                     float* norms, uint32_t* hist, const uint32_t* prev_packed,
+                     const float* prev_norms, void* stream);
+
+/* Level update (Algorithm 1 lines 2-7; Section 3.2, the minimisation after Eq. MQV with the
+ * CDF weights lambda_z = N_z^2 / sum N_z^2): for every layer with at least 3 levels, merge
+ * the num_samples histograms of that layer with those weights and minimise
+ * sum_j int_{l_j}^{l_{j+1}} (l_{j+1}-u)(u-l_j) dF~(u) by exact coordinate minimisation
+ * (the solver is this library's: the paper states the objective only).
+ *   hist dev [num_samples][L][LQ_HIST_STRIDE];  norms dev [num_samples][L].
+ * The new levels are staged: they take effect at the next lq_quantize_pack.  Layers with no
+ * usable mass keep their levels. */
+int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
+                  void* stream);
+
+/* DECODE + aggregate (Algorithm 1 lines 15 and 17): gbar = (1/K) sum_k N_k * sign * l_idx,
+ * summed in fp32 in worker order, with the levels of the latest lq_quantize_pack.
+ *   packed dev [K][W];  norms dev [K][L];  gbar dev [D_pad] out. */
+int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float* norms,
+                        float* gbar, void* stream);
+
+/* QODA state (Algorithm 1; Eq. ODA).  qoda_init sets Y_1 = 0, X_{3/2} = X_1, S_0 = 0,
+ * eta_1 = 1, t = 1 (initialisation V^_{k,1/2} = 0).   X1, Y, Xhalf dev [D_pad]. */
+int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stream);
+
+/* One QODA iteration after the workers' messages exist (Algorithm 1 lines 15-18 and line 10
+ * of the next iteration; Eq. ODA; Eq. general_stepsize):
+ *   S_t = S_{t-1} + (statistic left by the last lq_quantize_pack) / K^2,
+ *   eta_{t+1} = gamma_{t+1} = fp32((1 + S_t)^(-1/2)),
+ *   gbar = mean of the K decoded messages,  Y_{t+1} = Y_t - gbar,
+ *   X_{t+1} = fma(eta_{t+1}, Y_{t+1}, X_1),  X_{t+3/2} = fma(-gamma_{t+1}, gbar, X_{t+1}).
+ * One fused pass: each packed message is read once.
+ *   packed dev [K][W], norms dev [K][L], X1 dev [D_pad] in;  Y dev [D_pad] in/out;
+ *   Xhalf dev [D_pad] out (X_{t+3/2});  X_opt, gbar_opt: NULL or dev [D_pad] out. */
+int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1,
+              float* Y, float* Xhalf, float* X_opt, float* gbar_opt, void* stream);
+
+/* Host copies of the QODA scalars (t = index of the next iteration, S, eta); synchronises.
+ * Any output may be NULL. */
+int qoda_get_scalars(const lq_plan* plan, int64_t* t, double* S, double* eta);
+
+/* Per-(worker, layer) squared differences left by the last lq_quantize_pack
+ * (host_sq_diff [K][L] doubles) and status flags (host_flags [K][L], LQ_STATUS_*) of the
+ * last norm computation.  Either may be NULL.  Synchronises. */
+int lq_get_statistics(const lq_plan* plan, double* host_sq_diff, uint32_t* host_flags);
+
+const char* lq_error_string(int code);
+const char* lq_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQ_H_ */

@@ -101,8 +101,11 @@ float orc_layer_norm(const float* v, int64_t d, int q, int* status)
  *   idx = tau + up,  sign = sign bit of v.
  * `near` counts coordinates whose decision is within 1e-6 (relative to the interval)
  * of the threshold.  norm == 0 gives an all-zero message.
+ * v points at coordinate `first_index` of the layer and d coordinates are processed, so
+ * that a test can quantize a slice of a large layer.
  * ---------------------------------------------------------------------------------- */
-void orc_quantize_layer(const float* v, int64_t d, float norm, const float* level, int n,
+void orc_quantize_layer(const float* v, int64_t d, int64_t first_index, float norm,
+                        const float* level, int n,
                         uint64_t seed, uint32_t step, uint32_t worker, uint32_t layer,
                         uint8_t* idx, uint8_t* sign, int64_t* near)
 {
@@ -121,7 +124,7 @@ void orc_quantize_layer(const float* v, int64_t d, float norm, const float* leve
         for (int j = 1; j <= n - 2; ++j) if (level[j] <= u) tau = j;
         float num = u - level[tau];
         float den = level[tau + 1] - level[tau];
-        float rho = orc_uniform(seed, step, worker, layer, (uint64_t)i);
+        float rho = orc_uniform(seed, step, worker, layer, (uint64_t)(first_index + i));
         float t = rho * den;
         int up = (t < num) ? 1 : 0;
         if (fabsf(t - num) <= 1e-6f * den) ++near_count;

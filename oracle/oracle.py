@@ -43,7 +43,7 @@ def lib():
         L.orc_uniform.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64]
         L.orc_layer_norm.restype = C.c_float
         L.orc_layer_norm.argtypes = [f32p, C.c_int64, C.c_int, C.POINTER(C.c_int)]
-        L.orc_quantize_layer.argtypes = [f32p, C.c_int64, C.c_float, f32p, C.c_int, C.c_uint64,
+        L.orc_quantize_layer.argtypes = [f32p, C.c_int64, C.c_int64, C.c_float, f32p, C.c_int, C.c_uint64,
                                          C.c_uint32, C.c_uint32, C.c_uint32, u8p, u8p,
                                          C.POINTER(C.c_int64)]
         L.orc_round_up_probability.restype = C.c_double
@@ -97,11 +97,12 @@ def layer_norm(v: np.ndarray, q: int):
     return np.float32(n), st.value
 
 
-def quantize_layer(v, norm, levels, seed, step, worker, layer):
-    """Returns (idx u8[d], sign u8[d], near-threshold count)."""
+def quantize_layer(v, norm, levels, seed, step, worker, layer, first_index=0):
+    """Returns (idx u8[d], sign u8[d], near-threshold count) for coordinates
+    first_index .. first_index+len(v)-1 of the layer."""
     v = _f32(v); levels = _f32(levels)
     idx = np.zeros(v.size, np.uint8); sg = np.zeros(v.size, np.uint8); near = C.c_int64(0)
-    lib().orc_quantize_layer(_p(v, C.c_float), v.size, C.c_float(float(norm)), _p(levels, C.c_float),
+    lib().orc_quantize_layer(_p(v, C.c_float), v.size, first_index, C.c_float(float(norm)), _p(levels, C.c_float),
                              levels.size, seed, step, worker, layer, _p(idx, C.c_uint8),
                              _p(sg, C.c_uint8), C.byref(near))
     return idx, sg, near.value

@@ -1,0 +1,190 @@
+"""Thin ctypes binding of liblq.so: argument marshalling only.
+
+Every step of the hot path runs inside the CUDA library; this module only converts torch
+tensors to raw device pointers and passes the current CUDA stream.  Function names mirror
+the C entry points declared in include/lq.h.  There is no CPU fallback: if the library is
+missing, importing it raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblq.so")
+
+NUM_BINS = 386
+HIST_STRIDE = 512
+STATUS_ZERO_NORM = 1
+STATUS_NONFINITE = 2
+
+EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
+           "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
+           "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
+           "qoda_get_scalars", "lq_get_statistics", "lq_error_string", "lq_last_error"]
+
+
+class LqError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen liblq.so and declare the C signatures.  Raises if the library was not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise LqError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_14371_b200.build` "
+                      "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64, u32, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64
+    L.lq_plan_create.argtypes = [C.POINTER(vp), i32, C.POINTER(i64), C.POINTER(i32), i32, i32, u64]
+    L.lq_plan_destroy.argtypes = [vp]
+    L.lq_plan_padded_elems.argtypes = [vp]; L.lq_plan_padded_elems.restype = i64
+    L.lq_plan_packed_words.argtypes = [vp]; L.lq_plan_packed_words.restype = i64
+    L.lq_plan_layer_info.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+    L.lq_set_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
+    L.lq_get_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
+    L.lq_layer_norms.argtypes = [vp, vp, vp, vp]
+    L.lq_quantize_pack.argtypes = [vp, vp, u32, vp, vp, vp, vp, vp, vp]
+    L.lq_fit_levels.argtypes = [vp, vp, vp, i32, vp]
+    L.lq_decode_aggregate.argtypes = [vp, vp, vp, vp, vp]
+    L.qoda_init.argtypes = [vp, vp, vp, vp, vp]
+    L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
+    L.lq_error_string.argtypes = [C.c_int]; L.lq_error_string.restype = C.c_char_p
+    L.lq_last_error.argtypes = []; L.lq_last_error.restype = C.c_char_p
+    for name in EXPORTS:
+        getattr(L, name)              # raises AttributeError if the library lacks an entry point
+    _lib = L
+    return L
+
+
+def _check(code: int) -> None:
+    if code != 0:
+        L = load_library()
+        raise LqError(f"{L.lq_error_string(code).decode()} ({code}): {L.lq_last_error().decode()}")
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise LqError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise LqError(f"expected dtype {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Plan:
+    """Owns one lq_plan.  Methods carry the names of the C entry points."""
+
+    def __init__(self, layer_sizes: Sequence[int], bits, q: int, num_workers: int, seed: int):
+        L = load_library()
+        n = len(layer_sizes)
+        if isinstance(bits, int):
+            bits = [bits] * n
+        self.layer_sizes = [int(s) for s in layer_sizes]
+        self.bits = [int(b) for b in bits]
+        self.q, self.num_workers, self.seed = int(q), int(num_workers), int(seed)
+        sizes = (C.c_int64 * max(n, 1))(*self.layer_sizes)
+        bb = (C.c_int32 * max(n, 1))(*self.bits)
+        h = C.c_void_p()
+        _check(L.lq_plan_create(C.byref(h), n, sizes, bb, self.q, self.num_workers, C.c_uint64(self.seed)))
+        self._h = h
+        self.num_layers = n
+        self.padded_elems = int(L.lq_plan_padded_elems(h))
+        self.packed_words = int(L.lq_plan_packed_words(h))
+        self.elem_offsets: List[int] = []
+        self.word_offsets: List[int] = []
+        for m in range(n):
+            e, w, nl = C.c_int64(), C.c_int64(), C.c_int32()
+            _check(L.lq_plan_layer_info(h, m, C.byref(e), C.byref(w), C.byref(nl)))
+            self.elem_offsets.append(e.value); self.word_offsets.append(w.value)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            load_library().lq_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- levels -------------------------------------------------------------------------
+    def lq_set_levels(self, layer: int, levels) -> None:
+        arr = (C.c_float * len(levels))(*[float(x) for x in levels])
+        _check(load_library().lq_set_levels(self._h, layer, arr, len(levels)))
+
+    def lq_get_levels(self, layer: int) -> List[float]:
+        n = 1 << self.bits[layer]
+        arr = (C.c_float * n)()
+        _check(load_library().lq_get_levels(self._h, layer, arr, n))
+        return list(arr)
+
+    # ---- hot path -----------------------------------------------------------------------
+    def lq_layer_norms(self, grads: torch.Tensor, norms: torch.Tensor) -> None:
+        _check(load_library().lq_layer_norms(self._h, _ptr(grads, torch.float32), _ptr(norms, torch.float32),
+                                             _stream()))
+
+    def lq_quantize_pack(self, grads, step: int, packed, norms, hist=None, prev_packed=None,
+                         prev_norms=None) -> None:
+        _check(load_library().lq_quantize_pack(
+            self._h, _ptr(grads, torch.float32), C.c_uint32(step & 0xFFFFFFFF), _ptr(packed, torch.int32),
+            _ptr(norms, torch.float32), _ptr(hist, torch.int32), _ptr(prev_packed, torch.int32),
+            _ptr(prev_norms, torch.float32), _stream()))
+
+    def lq_fit_levels(self, hist, norms, num_samples: int) -> None:
+        _check(load_library().lq_fit_levels(self._h, _ptr(hist, torch.int32), _ptr(norms, torch.float32),
+                                            num_samples, _stream()))
+
+    def lq_decode_aggregate(self, packed, norms, gbar) -> None:
+        _check(load_library().lq_decode_aggregate(self._h, _ptr(packed, torch.int32), _ptr(norms, torch.float32),
+                                                  _ptr(gbar, torch.float32), _stream()))
+
+    def qoda_init(self, X1, Y, Xhalf) -> None:
+        _check(load_library().qoda_init(self._h, _ptr(X1, torch.float32), _ptr(Y, torch.float32),
+                                        _ptr(Xhalf, torch.float32), _stream()))
+
+    def qoda_step(self, packed, norms, X1, Y, Xhalf, X=None, gbar=None) -> None:
+        _check(load_library().qoda_step(self._h, _ptr(packed, torch.int32), _ptr(norms, torch.float32),
+                                        _ptr(X1, torch.float32), _ptr(Y, torch.float32),
+                                        _ptr(Xhalf, torch.float32), _ptr(X, torch.float32),
+                                        _ptr(gbar, torch.float32), _stream()))
+
+    def qoda_get_scalars(self):
+        t, S, eta = C.c_int64(), C.c_double(), C.c_double()
+        _check(load_library().qoda_get_scalars(self._h, C.byref(t), C.byref(S), C.byref(eta)))
+        return t.value, S.value, eta.value
+
+    def lq_get_statistics(self):
+        """Returns (sq_diff [K][L] float64, status [K][L] int) as torch CPU tensors."""
+        K, Ln = self.num_workers, max(self.num_layers, 1)
+        sq = (C.c_double * (K * Ln))(); fl = (C.c_uint32 * (K * Ln))()
+        _check(load_library().lq_get_statistics(self._h, sq, fl))
+        return (torch.tensor(list(sq), dtype=torch.float64).view(K, Ln)[:, : self.num_layers],
+                torch.tensor(list(fl), dtype=torch.int64).view(K, Ln)[:, : self.num_layers])
+
+    # ---- allocation helpers (device memory only; no arithmetic) ----------------------------
+    def empty_packed(self, device="cuda") -> torch.Tensor:
+        return torch.empty((self.num_workers, max(self.packed_words, 1)), dtype=torch.int32, device=device)
+
+    def empty_norms(self, device="cuda") -> torch.Tensor:
+        return torch.empty((self.num_workers, max(self.num_layers, 1)), dtype=torch.float32, device=device)
+
+    def zero_hist(self, device="cuda") -> torch.Tensor:
+        return torch.zeros((self.num_workers, max(self.num_layers, 1), HIST_STRIDE), dtype=torch.int32,
+                           device=device)

@@ -1,0 +1,346 @@
+// Host side of liblq: the plan object and the extern "C" entry points declared in lq.h.
+// No kernel lives here; this file validates arguments, owns the plan's device tables and
+// enqueues the launchers of the other translation units on the caller's stream.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "lq_internal.cuh"
+
+using namespace lq;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define LQ_CUDA(expr)                                                                         \
+    do {                                                                                      \
+        cudaError_t e_ = (expr);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail(e_ == cudaErrorMemoryAllocation ? LQ_ENOMEM : LQ_ECUDA, "%s: %s", #expr, \
+                        cudaGetErrorString(e_));                                              \
+    } while (0)
+
+}  // namespace
+
+// The three level tables: `stage` receives lq_set_levels / lq_fit_levels; at the next
+// lq_quantize_pack a changed stage is copied into the encode table that is not in use, which
+// becomes current, while the other keeps the levels of the previous message.
+struct lq_plan {
+    PlanDev dev{};
+    std::vector<LayerDesc> layers;
+    std::vector<Tile> tiles;
+    int device = 0;
+    uint64_t seed = 0;
+    LayerDesc* d_layers = nullptr;
+    Tile* d_tiles = nullptr;
+    float* d_levels_stage = nullptr;
+    float* d_levels_enc[2] = {nullptr, nullptr};
+    int cur = 0, prev = 0;
+    bool stage_dirty = false;
+    bool have_message = false;
+    bool qoda_ready = false;
+    bool stat_pending = false;
+};
+
+namespace {
+
+void free_plan(lq_plan* p)
+{
+    if (!p) return;
+    cudaFree(p->d_layers); cudaFree(p->d_tiles);
+    cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
+    cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars);
+    delete p;
+}
+
+template <typename T>
+cudaError_t dev_alloc_zero(T** ptr, size_t count)
+{
+    const size_t bytes = (count ? count : 1) * sizeof(T);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(ptr), bytes);
+    if (e != cudaSuccess) { *ptr = nullptr; return e; }
+    return cudaMemset(*ptr, 0, bytes);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* lq_last_error(void) { return g_err; }
+
+const char* lq_error_string(int code)
+{
+    switch (code) {
+        case LQ_OK: return "ok";
+        case LQ_EINVAL: return "invalid argument";
+        case LQ_ENOMEM: return "out of memory";
+        case LQ_ECUDA: return "CUDA runtime error";
+        case LQ_ESTATE: return "call out of order";
+        default: return "unknown error";
+    }
+}
+
+int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes, const int32_t* bits,
+                   int32_t q, int32_t num_workers, uint64_t seed)
+{
+    if (!out) return fail(LQ_EINVAL, "out is NULL");
+    *out = nullptr;
+    if (num_layers < 0 || (num_layers > 0 && (!layer_sizes || !bits)))
+        return fail(LQ_EINVAL, "num_layers < 0 or NULL layer arrays");
+    if (q < 0 || q > 16) return fail(LQ_EINVAL, "q must be 0 (infinity norm) or 1..16, got %d", q);
+    if (num_workers < 1 || num_workers > LQ_MAX_WORKERS)
+        return fail(LQ_EINVAL, "num_workers must be in [1, %d], got %d", LQ_MAX_WORKERS, num_workers);
+
+    lq_plan* p = new (std::nothrow) lq_plan;
+    if (!p) return fail(LQ_ENOMEM, "host allocation failed");
+    int64_t elem = 0, word = 0, ntiles = 0;
+    try {
+        p->layers.resize((size_t)num_layers);
+        for (int m = 0; m < num_layers; ++m) {
+            const int64_t d = layer_sizes[m];
+            const int b = bits[m];
+            if (d < 0 || d >= ((int64_t)1 << 31)) { delete p; return fail(LQ_EINVAL, "layer %d: size %lld out of [0, 2^31)", m, (long long)d); }
+            if (b < 1 || b > LQ_MAX_BITS) { delete p; return fail(LQ_EINVAL, "layer %d: bits %d out of [1, %d]", m, b, LQ_MAX_BITS); }
+            LayerDesc& L = p->layers[(size_t)m];
+            L.elem_off = elem; L.word_off = word; L.size = d; L.bits = b; L.nlevels = 1 << b;
+            L.nblocks = (int32_t)((d + kBlockCoords - 1) / kBlockCoords);
+            L.first_tile = (int32_t)ntiles;
+            L.ntiles = (L.nblocks + kTileBlocks - 1) / kTileBlocks;
+            L.pad_ = 0;
+            for (int t = 0; t < L.ntiles; ++t) {
+                Tile tl;
+                tl.layer = m; tl.block0 = t * kTileBlocks;
+                tl.nblocks = L.nblocks - tl.block0 < kTileBlocks ? L.nblocks - tl.block0 : kTileBlocks;
+                tl.pad_ = 0;
+                p->tiles.push_back(tl);
+            }
+            ntiles += L.ntiles;
+            if (ntiles >= ((int64_t)1 << 31) - 1) { delete p; return fail(LQ_EINVAL, "too many tiles"); }
+            elem += (d + 31) / 32 * 32;
+            word += (int64_t)L.nblocks * 32 * (b + 1);
+        }
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return fail(LQ_ENOMEM, "host allocation failed");
+    }
+    if (elem == 0) elem = 32;
+    p->seed = seed;
+    PlanDev& d = p->dev;
+    d.num_layers = num_layers; d.num_tiles = (int32_t)ntiles; d.num_workers = num_workers; d.q = q;
+    d.padded_elems = elem; d.packed_words = word;
+    d.seed_lo = (uint32_t)seed; d.seed_hi = (uint32_t)(seed >> 32);
+
+    cudaError_t e = cudaGetDevice(&p->device);
+    const size_t KL = (size_t)num_workers * (size_t)(num_layers ? num_layers : 1);
+    const size_t KT = (size_t)num_workers * (size_t)(ntiles ? ntiles : 1);
+    const size_t lev = (size_t)(num_layers ? num_layers : 1) * kLevelStride;
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_layers, p->layers.size());
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_tiles, p->tiles.size());
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_stage, lev);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[0], lev);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[1], lev);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.stat_partial, KT);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.scalars, 1);
+    if (e == cudaSuccess && !p->layers.empty())
+        e = cudaMemcpy(p->d_layers, p->layers.data(), p->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && !p->tiles.empty())
+        e = cudaMemcpy(p->d_tiles, p->tiles.data(), p->tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        // uniform levels j / (2^b - 1), rounded once from fp64
+        std::vector<float> host(lev, 0.0f);
+        for (int m = 0; m < num_layers; ++m) {
+            const int n = p->layers[(size_t)m].nlevels;
+            for (int j = 0; j < n; ++j)
+                host[(size_t)m * kLevelStride + j] = (float)((double)j / (double)(n - 1));
+        }
+        for (float* t : {p->d_levels_stage, p->d_levels_enc[0], p->d_levels_enc[1]})
+            if (e == cudaSuccess) e = cudaMemcpy(t, host.data(), lev * sizeof(float), cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) {
+        QodaScalars s0{0.0, 0.0, 1, 1.0f, 0.0f};
+        e = cudaMemcpy(d.scalars, &s0, sizeof s0, cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        const int code = e == cudaErrorMemoryAllocation ? LQ_ENOMEM : LQ_ECUDA;
+        free_plan(p);
+        return fail(code, "plan setup: %s", cudaGetErrorString(e));
+    }
+    d.layers = p->d_layers; d.tiles = p->d_tiles;
+    *out = p;
+    return LQ_OK;
+}
+
+int lq_plan_destroy(lq_plan* plan)
+{
+    if (!plan) return LQ_OK;
+    cudaDeviceSynchronize();
+    free_plan(plan);
+    return LQ_OK;
+}
+
+int64_t lq_plan_padded_elems(const lq_plan* plan) { return plan ? plan->dev.padded_elems : (int64_t)fail(LQ_EINVAL, "plan is NULL"); }
+int64_t lq_plan_packed_words(const lq_plan* plan) { return plan ? plan->dev.packed_words : (int64_t)fail(LQ_EINVAL, "plan is NULL"); }
+
+int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, int64_t* word_off, int32_t* num_levels)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    if (layer < 0 || layer >= plan->dev.num_layers) return fail(LQ_EINVAL, "layer %d out of range", layer);
+    const LayerDesc& L = plan->layers[(size_t)layer];
+    if (elem_off) *elem_off = L.elem_off;
+    if (word_off) *word_off = L.word_off;
+    if (num_levels) *num_levels = L.nlevels;
+    return LQ_OK;
+}
+
+int lq_set_levels(lq_plan* plan, int32_t layer, const float* host_levels, int32_t n)
+{
+    if (!plan || !host_levels) return fail(LQ_EINVAL, "NULL argument");
+    if (layer < 0 || layer >= plan->dev.num_layers) return fail(LQ_EINVAL, "layer %d out of range", layer);
+    const LayerDesc& L = plan->layers[(size_t)layer];
+    if (n != L.nlevels) return fail(LQ_EINVAL, "layer %d has %d levels, got %d", layer, L.nlevels, n);
+    if (host_levels[0] != 0.0f || host_levels[n - 1] != 1.0f)
+        return fail(LQ_EINVAL, "levels must start at 0 and end at 1");
+    for (int j = 1; j < n; ++j) {
+        // gaps below 2^-100 are refused: they could not be told apart from rounding noise anyway
+        if (!(host_levels[j] - host_levels[j - 1] >= 7.888609052210118e-31f))
+            return fail(LQ_EINVAL, "levels must be strictly increasing (index %d)", j);
+    }
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(plan->d_levels_stage + (size_t)layer * kLevelStride, host_levels,
+                       (size_t)n * sizeof(float), cudaMemcpyHostToDevice));
+    plan->stage_dirty = true;
+    return LQ_OK;
+}
+
+int lq_get_levels(const lq_plan* plan, int32_t layer, float* host_levels, int32_t n)
+{
+    if (!plan || !host_levels) return fail(LQ_EINVAL, "NULL argument");
+    if (layer < 0 || layer >= plan->dev.num_layers) return fail(LQ_EINVAL, "layer %d out of range", layer);
+    const LayerDesc& L = plan->layers[(size_t)layer];
+    if (n != L.nlevels) return fail(LQ_EINVAL, "layer %d has %d levels, got %d", layer, L.nlevels, n);
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(host_levels, plan->d_levels_stage + (size_t)layer * kLevelStride,
+                       (size_t)n * sizeof(float), cudaMemcpyDeviceToHost));
+    return LQ_OK;
+}
+
+int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream)
+{
+    if (!plan || !grads || !norms) return fail(LQ_EINVAL, "NULL argument");
+    if (plan->dev.num_layers == 0) return LQ_OK;
+    LQ_CUDA(launch_norm(plan->dev, grads, norms, (cudaStream_t)stream));
+    return LQ_OK;
+}
+
+int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t* packed, float* norms,
+                     uint32_t* hist, const uint32_t* prev_packed, const float* prev_norms, void* stream)
+{
+    if (!plan || !grads || !packed || !norms) return fail(LQ_EINVAL, "NULL argument");
+    if ((prev_packed == nullptr) != (prev_norms == nullptr))
+        return fail(LQ_EINVAL, "prev_packed and prev_norms must both be given or both be NULL");
+    if (prev_packed == packed) return fail(LQ_EINVAL, "prev_packed must not alias packed");
+    if (plan->dev.num_layers == 0) return LQ_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t lev_bytes = (size_t)plan->dev.num_layers * kLevelStride * sizeof(float);
+    if (plan->stage_dirty) {
+        const int next = plan->have_message ? 1 - plan->cur : plan->cur;
+        LQ_CUDA(cudaMemcpyAsync(plan->d_levels_enc[next], plan->d_levels_stage, lev_bytes,
+                                cudaMemcpyDeviceToDevice, s));
+        plan->prev = plan->cur;
+        plan->cur = next;
+        plan->stage_dirty = false;
+    } else {
+        plan->prev = plan->cur;
+    }
+    LQ_CUDA(launch_norm(plan->dev, grads, norms, s));
+    LQ_CUDA(launch_quantize(plan->dev, grads, step, packed, norms, hist, prev_packed, prev_norms,
+                            plan->d_levels_enc[plan->cur], plan->d_levels_enc[plan->prev], s));
+    plan->have_message = true;
+    plan->stat_pending = true;
+    return LQ_OK;
+}
+
+int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples, void* stream)
+{
+    if (!plan || !hist || !norms) return fail(LQ_EINVAL, "NULL argument");
+    if (num_samples < 1 || num_samples > LQ_MAX_WORKERS)
+        return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
+    LQ_CUDA(launch_fit(plan->dev, hist, norms, num_samples, plan->d_levels_stage, (cudaStream_t)stream));
+    plan->stage_dirty = true;
+    return LQ_OK;
+}
+
+int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float* norms, float* gbar, void* stream)
+{
+    if (!plan || !packed || !norms || !gbar) return fail(LQ_EINVAL, "NULL argument");
+    LQ_CUDA(launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], nullptr, nullptr, nullptr,
+                          nullptr, gbar, false, (cudaStream_t)stream));
+    return LQ_OK;
+}
+
+int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stream)
+{
+    if (!plan || !X1 || !Y || !Xhalf) return fail(LQ_EINVAL, "NULL argument");
+    LQ_CUDA(launch_qoda_init(plan->dev, X1, Y, Xhalf, (cudaStream_t)stream));
+    plan->qoda_ready = true;
+    plan->stat_pending = false;
+    return LQ_OK;
+}
+
+int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1, float* Y,
+              float* Xhalf, float* X_opt, float* gbar_opt, void* stream)
+{
+    if (!plan || !packed || !norms || !X1 || !Y || !Xhalf) return fail(LQ_EINVAL, "NULL argument");
+    if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
+    if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
+    cudaStream_t s = (cudaStream_t)stream;
+    LQ_CUDA(launch_qoda_scalars(plan->dev, s));
+    LQ_CUDA(launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
+                          gbar_opt, true, s));
+    plan->stat_pending = false;
+    return LQ_OK;
+}
+
+int qoda_get_scalars(const lq_plan* plan, int64_t* t, double* S, double* eta)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    QodaScalars h;
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(&h, plan->dev.scalars, sizeof h, cudaMemcpyDeviceToHost));
+    if (t) *t = (int64_t)h.t;
+    if (S) *S = h.S;
+    if (eta) *eta = (double)h.eta;
+    return LQ_OK;
+}
+
+int lq_get_statistics(const lq_plan* plan, double* host_sq_diff, uint32_t* host_flags)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    const size_t KL = (size_t)plan->dev.num_workers * (size_t)plan->dev.num_layers;
+    LQ_CUDA(cudaDeviceSynchronize());
+    if (host_sq_diff && KL)
+        LQ_CUDA(cudaMemcpy(host_sq_diff, plan->dev.sq_diff, KL * sizeof(double), cudaMemcpyDeviceToHost));
+    if (host_flags && KL)
+        LQ_CUDA(cudaMemcpy(host_flags, plan->dev.status, KL * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return LQ_OK;
+}
+
+}  // extern "C"

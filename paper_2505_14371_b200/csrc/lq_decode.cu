@@ -1,0 +1,188 @@
+// DECODE + aggregate of the K workers' messages, alone or fused with the optimistic dual averaging
+// update (Algorithm 1 lines 15-18 and line 10 of the next iteration; Eq. ODA; Eq. general_stepsize).
+//
+// One CTA per tile (up to 8 blocks of 1024 coordinates of one layer), one warp per block.  A lane
+// owns the same 32 coordinates it owned at encode time, so it reads (b+1) words per worker with
+// 128-byte coalesced warp loads, looks the decoded values up in a per-(worker, layer) table in shared
+// memory, sums them in worker order in registers, and finishes with float4 reads of Y and X_1 and
+// float4 writes of Y and X_{t+3/2}.  Every packed word and every state element is touched once.
+#include "lq_internal.cuh"
+
+namespace lq {
+
+constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
+
+template <int B>
+__device__ __forceinline__ uint32_t code_at(const uint32_t (&cw)[B], int p)
+{
+    const int off = p * B, w = off >> 5, s = off & 31;
+    uint32_t v = cw[w] >> s;
+    if (s + B > 32) v |= cw[w + 1] << (32 - s);
+    return v & ((1u << B) - 1u);
+}
+
+template <int B>
+__device__ __forceinline__ void decode_accumulate(float (&acc)[32], const uint32_t* __restrict__ words,
+                                                  const float* __restrict__ table)
+{
+    const uint32_t signw = words[0];
+    uint32_t cw[B];
+#pragma unroll
+    for (int w = 0; w < B; ++w) cw[w] = words[(w + 1) * 32];
+#pragma unroll
+    for (int p = 0; p < 32; ++p) {
+        const uint32_t mag = __float_as_uint(table[code_at<B>(cw, p)]);
+        acc[p] += __uint_as_float(mag ^ ((signw >> p) << 31));
+    }
+}
+
+struct DecodeArgs {
+    const uint32_t* packed;
+    const float* norms;
+    const float* levels;
+    const float* X1;
+    float* Y;
+    float* Xhalf;
+    float* X;
+    float* gbar;
+};
+
+// Any worker count: the accumulators live across chunks of kWorkerChunk workers.
+template <int B, bool kQoda>
+__device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
+                                                     int64_t blk, bool active, const DecodeArgs& a,
+                                                     float (*table)[kMaxLevels], float eta)
+{
+    const int lane = threadIdx.x & 31;
+    const int K = p.num_workers;
+    const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
+    float acc[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
+
+    for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
+        const int kc = min(kWorkerChunk, K - k0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < kc * L.nlevels; i += blockDim.x) {
+            const int kk = i / L.nlevels, j = i - kk * L.nlevels;
+            table[kk][j] = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
+                                     a.levels[(int64_t)layer * kLevelStride + j]);
+        }
+        __syncthreads();
+        if (active)
+            for (int kk = 0; kk < kc; ++kk)
+                decode_accumulate<B>(acc, a.packed + (int64_t)(k0 + kk) * p.packed_words + woff, table[kk]);
+    }
+    if (!active) return;
+
+    const float invK = __fdiv_rn(1.0f, (float)K);
+    const int64_t base = L.elem_off + blk * kBlockCoords + 4 * lane;
+    const int64_t limit = L.elem_off + L.size;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int64_t pos = base + 128 * j;
+        if (pos >= limit) continue;
+        float4 g;
+        g.x = __fmul_rn(acc[4 * j + 0], invK);
+        g.y = __fmul_rn(acc[4 * j + 1], invK);
+        g.z = __fmul_rn(acc[4 * j + 2], invK);
+        g.w = __fmul_rn(acc[4 * j + 3], invK);
+        if (a.gbar) *reinterpret_cast<float4*>(a.gbar + pos) = g;
+        if (kQoda) {
+            const float4 y0 = *reinterpret_cast<const float4*>(a.Y + pos);
+            const float4 x1 = __ldg(reinterpret_cast<const float4*>(a.X1 + pos));
+            float4 y, x, h;
+            y.x = __fsub_rn(y0.x, g.x); y.y = __fsub_rn(y0.y, g.y);
+            y.z = __fsub_rn(y0.z, g.z); y.w = __fsub_rn(y0.w, g.w);
+            x.x = fmaf(eta, y.x, x1.x); x.y = fmaf(eta, y.y, x1.y);
+            x.z = fmaf(eta, y.z, x1.z); x.w = fmaf(eta, y.w, x1.w);
+            h.x = fmaf(-eta, g.x, x.x); h.y = fmaf(-eta, g.y, x.y);
+            h.z = fmaf(-eta, g.z, x.z); h.w = fmaf(-eta, g.w, x.w);
+            *reinterpret_cast<float4*>(a.Y + pos) = y;
+            *reinterpret_cast<float4*>(a.Xhalf + pos) = h;
+            if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
+        }
+    }
+}
+
+template <bool kQoda>
+__global__ void __launch_bounds__(kThreads) decode_kernel(PlanDev p, DecodeArgs a)
+{
+    __shared__ float table[kWorkerChunk][kMaxLevels];
+    const Tile tile = p.tiles[blockIdx.x];
+    const int layer = tile.layer;
+    const LayerDesc L = p.layers[layer];
+    const int warp = threadIdx.x >> 5;
+    const bool active = warp < tile.nblocks;
+    const int64_t blk = tile.block0 + warp;
+    const float eta = kQoda ? p.scalars->eta : 0.0f;
+
+    switch (L.bits) {
+#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kQoda>(p, L, layer, blk, active, a, table, eta); break;
+        LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
+#undef LQ_CASE
+        default: break;
+    }
+}
+
+// S_t = S_{t-1} + (sum over workers and layers of the squared differences) / K^2,
+// eta_{t+1} = fp32((1 + S_t)^(-1/2)); one CTA, fixed summation order.
+__global__ void __launch_bounds__(256) qoda_scalars_kernel(PlanDev p)
+{
+    __shared__ double scratch[8];
+    const int n = p.num_workers * p.num_layers;
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) acc += p.sq_diff[i];
+    const double total = block_reduce<false>(acc, scratch);
+    if (threadIdx.x == 0) {
+        QodaScalars* q = p.scalars;
+        const double K = (double)p.num_workers;
+        const double delta = total / (K * K);
+        q->last_delta = delta;
+        q->S = q->S + delta;
+        q->eta = (float)(1.0 / sqrt(1.0 + q->S));
+        q->t = q->t + 1;
+    }
+}
+
+__global__ void qoda_init_kernel(PlanDev p, const float* __restrict__ X1, float* __restrict__ Y,
+                                 float* __restrict__ Xhalf)
+{
+    const int64_t n4 = p.padded_elems / 4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        reinterpret_cast<float4*>(Y)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4*>(Xhalf)[i] = reinterpret_cast<const float4*>(X1)[i];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        QodaScalars* q = p.scalars;
+        q->S = 0.0; q->last_delta = 0.0; q->t = 1; q->eta = 1.0f;
+    }
+}
+
+cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
+                          const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
+                          float* gbar, bool qoda, cudaStream_t s)
+{
+    if (p.num_tiles == 0) return cudaSuccess;
+    DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
+    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles, kThreads, 0, s>>>(p, a);
+    else      decode_kernel<false><<<(unsigned)p.num_tiles, kThreads, 0, s>>>(p, a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s)
+{
+    qoda_scalars_kernel<<<1, 256, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_qoda_init(const PlanDev& p, const float* X1, float* Y, float* Xhalf, cudaStream_t s)
+{
+    const int64_t n4 = p.padded_elems / 4;
+    const unsigned blocks = (unsigned)((n4 + 255) / 256 < 148 * 8 ? (n4 + 255) / 256 + 1 : 148 * 8);
+    qoda_init_kernel<<<blocks, 256, 0, s>>>(p, X1, Y, Xhalf);
+    return cudaGetLastError();
+}
+
+}  // namespace lq

@@ -1,0 +1,185 @@
+// Level update (Algorithm 1 lines 2-7): for each layer, merge the sampled histograms with the
+// weights lambda_z = N_z^2 / sum N_z^2 and minimise
+//     sum_j int_{l_j}^{l_{j+1}} (l_{j+1} - u)(u - l_j) dF~(u)
+// (Section 3.2 of the paper, the minimisation that follows Eq. MQV).  The paper gives the objective
+// only; the solver is exact coordinate minimisation: with neighbours a < c fixed, the optimal level
+// l solves  F~(l) = F~(c) - int_a^c (u - a)/(c - a) dF~(u).  F~ is piecewise linear (uniform density
+// inside a histogram bin), so F~, its first moment and its inverse are closed forms.
+//
+// One CTA per layer; odd and even interior levels are updated in two parallel half-sweeps (levels of
+// one parity only depend on the other parity).  All arithmetic is fp64 and this file is compiled
+// without FMA contraction so that the sequence of roundings is the plain one.
+#include "lq_internal.cuh"
+
+namespace lq {
+
+constexpr int kBins = 385;            // bins 0..384 carry density; bin 385 (u = 1) never adds variance
+constexpr int kFitThreads = 128;
+constexpr int kMaxSweeps = 100;
+
+struct FitSmem {
+    double e[kBins + 1];
+    double mass[kBins];
+    double F[kBins + 1];
+    double M1[kBins + 1];
+    double l[kMaxLevels];
+    double lambda[LQ_MAX_WORKERS];
+    double red[kFitThreads / 32];
+    double moved;
+    int ok;
+};
+
+__device__ __forceinline__ double bin_edge(int i)
+{
+    if (i <= 0) return 0.0;
+    const int o = (i - 1) >> 4, m = (i - 1) & 15;
+    return ldexp(1.0 + (double)m * 0.0625, o - 24);
+}
+
+__device__ int bin_of(const FitSmem& s, double x)
+{
+    int lo = 0, hi = kBins - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s.e[mid] <= x) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__device__ double cdf(const FitSmem& s, double x, double* m1)
+{
+    const int i = bin_of(s, x);
+    double theta = (x - s.e[i]) / (s.e[i + 1] - s.e[i]);
+    if (theta > 1.0) theta = 1.0;
+    const double part = s.mass[i] * theta;
+    *m1 = s.M1[i] + part * ((s.e[i] + x) * 0.5);
+    return s.F[i] + part;
+}
+
+__device__ double cdf_inv(const FitSmem& s, double y)
+{
+    int lo = 0, hi = kBins;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (s.F[mid + 1] > y) hi = mid; else lo = mid + 1;
+    }
+    if (lo >= kBins) return 1.0;
+    double t = (y - s.F[lo]) / s.mass[lo];
+    if (t < 0.0) t = 0.0;
+    return s.e[lo] + t * (s.e[lo + 1] - s.e[lo]);
+}
+
+__global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, const uint32_t* __restrict__ hist,
+                                                                 const float* __restrict__ norms, int Z,
+                                                                 float* __restrict__ levels_stage)
+{
+    __shared__ FitSmem s;
+    const int m = blockIdx.x;
+    const LayerDesc L = p.layers[m];
+    const int n = L.nlevels;
+    if (n < 3 || L.size <= 0) return;
+    const int tid = threadIdx.x;
+
+    if (tid == 0) {
+        double wsum = 0.0;
+        for (int z = 0; z < Z; ++z) {
+            const double w = (double)norms[(int64_t)z * p.num_layers + m];
+            wsum += w * w;
+        }
+        s.ok = wsum > 0.0;
+        if (s.ok)
+            for (int z = 0; z < Z; ++z) {
+                const double w = (double)norms[(int64_t)z * p.num_layers + m];
+                s.lambda[z] = (w * w) / wsum;
+            }
+    }
+    __syncthreads();
+    if (!s.ok) return;
+
+    for (int i = tid; i <= kBins; i += kFitThreads) s.e[i] = bin_edge(i);
+    for (int i = tid; i < kBins; i += kFitThreads) {
+        double acc = 0.0;
+        for (int z = 0; z < Z; ++z)
+            acc += s.lambda[z] * (double)hist[((int64_t)z * p.num_layers + m) * LQ_HIST_STRIDE + i];
+        s.mass[i] = acc / (double)L.size;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        s.F[0] = 0.0; s.M1[0] = 0.0;
+        for (int i = 0; i < kBins; ++i) {
+            s.F[i + 1] = s.F[i] + s.mass[i];
+            s.M1[i + 1] = s.M1[i] + s.mass[i] * ((s.e[i] + s.e[i + 1]) * 0.5);
+        }
+        s.ok = (s.F[kBins] - s.mass[0]) > 0.0;
+    }
+    __syncthreads();
+    if (!s.ok) return;
+
+    const double above = s.F[kBins] - s.mass[0];
+    for (int j = tid; j < n; j += kFitThreads) {
+        if (j == 0) s.l[j] = 0.0;
+        else if (j == n - 1) s.l[j] = 1.0;
+        else s.l[j] = cdf_inv(s, s.mass[0] + above * ((double)j / (double)(n - 1)));
+    }
+    __syncthreads();
+
+    for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+        double moved = 0.0;
+        for (int parity = 1; parity >= 0; --parity) {
+            for (int j = tid; j <= n - 2; j += kFitThreads) {
+                if (j < 1 || (j & 1) != parity) continue;
+                const double a = s.l[j - 1], c = s.l[j + 1];
+                if (!(c > a)) continue;
+                double m1a, m1c, b;
+                const double Fa = cdf(s, a, &m1a), Fc = cdf(s, c, &m1c);
+                const double mass_ac = Fc - Fa;
+                if (!(mass_ac > 0.0)) b = (a + c) * 0.5;
+                else {
+                    const double target = Fc - ((m1c - m1a) - a * mass_ac) / (c - a);
+                    b = cdf_inv(s, target);
+                    if (b < a) b = a;
+                    if (b > c) b = c;
+                }
+                const double rel = fabs(b - s.l[j]) / (fabs(b) > 1e-300 ? fabs(b) : 1e-300);
+                if (rel > moved) moved = rel;
+                s.l[j] = b;
+            }
+            __syncthreads();
+        }
+        moved = warp_max(moved);
+        if ((tid & 31) == 0) s.red[tid >> 5] = moved;
+        __syncthreads();
+        if (tid == 0) {
+            double mx = s.red[0];
+            for (int w = 1; w < kFitThreads / 32; ++w) mx = fmax(mx, s.red[w]);
+            s.moved = mx;
+        }
+        __syncthreads();
+        if (s.moved <= 1e-13) break;
+    }
+
+    // round to fp32; force strict monotonicity by single-ulp steps (serial: order matters)
+    if (tid == 0) {
+        float* out = levels_stage + (int64_t)m * kLevelStride;
+        out[0] = 0.0f; out[n - 1] = 1.0f;
+        for (int j = 1; j <= n - 2; ++j) {
+            const float f = (float)s.l[j];
+            const float fl = nextafterf(out[j - 1], 2.0f);
+            out[j] = f > fl ? f : fl;
+        }
+        for (int j = n - 2; j >= 1; --j) {
+            const float ce = nextafterf(out[j + 1], -1.0f);
+            if (out[j] > ce) out[j] = ce;
+        }
+    }
+}
+
+cudaError_t launch_fit(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
+                       float* levels_stage, cudaStream_t s)
+{
+    if (p.num_layers == 0) return cudaSuccess;
+    fit_levels_kernel<<<(unsigned)p.num_layers, kFitThreads, 0, s>>>(p, hist, norms, num_samples, levels_stage);
+    return cudaGetLastError();
+}
+
+}  // namespace lq

@@ -1,0 +1,139 @@
+// Internal declarations shared by the .cu files of liblq (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lq.h"
+
+namespace lq {
+
+constexpr int kBlockCoords = 1024;    // coordinates per message block (32 lanes x 32 positions)
+constexpr int kTileBlocks = 8;        // blocks per tile = one per warp of a 256-thread CTA
+constexpr int kThreads = 256;
+constexpr int kLevelStride = 256;     // floats per layer in a level table
+constexpr int kMaxLevels = 256;
+
+struct LayerDesc {
+    int64_t elem_off;     // first element of the layer inside a worker's fp32 row
+    int64_t word_off;     // first word of the layer inside a worker's message
+    int64_t size;         // d_m
+    int32_t bits;         // b_m
+    int32_t nlevels;      // 2^b_m
+    int32_t nblocks;      // ceil(d_m / 1024)
+    int32_t first_tile;   // tiles of one layer are contiguous in the tile table
+    int32_t ntiles;
+    int32_t pad_;
+};
+
+struct Tile {
+    int32_t layer;
+    int32_t block0;       // first block of the tile inside its layer
+    int32_t nblocks;      // 1..kTileBlocks
+    int32_t pad_;
+};
+
+struct QodaScalars {
+    double S;             // running sum of Eq. (general_stepsize)
+    double last_delta;    // the term added by the last qoda_step
+    long long t;          // index of the next iteration
+    float eta;            // eta_t = gamma_t
+    float pad_;
+};
+
+// Device-side view of a plan, passed to kernels by value.
+struct PlanDev {
+    const LayerDesc* layers;
+    const Tile* tiles;
+    int32_t num_layers;
+    int32_t num_tiles;
+    int32_t num_workers;
+    int32_t q;            // 0 = infinity norm
+    int64_t padded_elems; // D_pad
+    int64_t packed_words; // W
+    uint32_t seed_lo, seed_hi;
+    double* norm_partial; // [K][num_tiles]
+    double* stat_partial; // [K][num_tiles]
+    double* sq_diff;      // [K][L]
+    float* rnorm;         // [K][L]   1/N, or 0 for a zeroed layer
+    uint32_t* status;     // [K][L]
+    QodaScalars* scalars;
+};
+
+struct lq_plan_impl;
+
+// ---- launchers (each enqueues on `s` and returns the launch status) ----
+cudaError_t launch_norm(const PlanDev& p, const float* grads, float* norms, cudaStream_t s);
+cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
+                            const float* norms, uint32_t* hist, const uint32_t* prev_packed,
+                            const float* prev_norms, const float* levels_cur,
+                            const float* levels_prev, cudaStream_t s);
+cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
+                          const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
+                          float* gbar, bool qoda, cudaStream_t s);
+cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s);
+cudaError_t launch_qoda_init(const PlanDev& p, const float* X1, float* Y, float* Xhalf,
+                             cudaStream_t s);
+cudaError_t launch_fit(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
+                       float* levels_stage, cudaStream_t s);
+
+// ---- device helpers ----
+#ifdef __CUDACC__
+
+// Philox4x32-10 (Salmon et al., SC'11): 10 rounds of two 32x32->64 multiplies and xors,
+// the key bumped by the Weyl constants between rounds.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_max(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Sum over the CTA in a fixed order (xor tree inside a warp, warps added in index order).
+// The result is valid in thread 0.  `scratch` holds one double per warp.
+template <bool kMax>
+__device__ __forceinline__ double block_reduce(double v, double* scratch)
+{
+    v = kMax ? warp_max(v) : warp_sum(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    double r = 0.0;
+    if (threadIdx.x == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        r = scratch[0];
+        for (int w = 1; w < nw; ++w) r = kMax ? fmax(r, scratch[w]) : r + scratch[w];
+    }
+    return r;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace lq

@@ -1,0 +1,132 @@
+// Per-layer L^q norms of K workers' gradients (Section 2.2 of the paper: v is represented by
+// (||v||_q, sign, u)).  Two launches: a streaming pass that leaves one fp64 partial per
+// (worker, tile), and a small pass that adds a layer's partials in a fixed order, so the
+// result does not depend on scheduling.
+#include "lq_internal.cuh"
+
+namespace lq {
+
+// mode 0: max |v|   1: sum |v|   2: sum v^2   3: sum |v|^q (integer q >= 3)
+template <int kMode>
+__device__ __forceinline__ void accumulate(double& acc, uint32_t& maxbits, float v, int q)
+{
+    if (kMode == 0) {
+        // |v| as an unsigned integer orders like the float; NaN and Inf have the largest patterns
+        const uint32_t b = __float_as_uint(v) & 0x7fffffffu;
+        maxbits = max(maxbits, b);
+    } else if (kMode == 1) {
+        acc += (double)fabsf(v);
+    } else if (kMode == 2) {
+        const double a = (double)v;
+        acc = fma(a, a, acc);            // the product of two floats is exact in fp64
+    } else {
+        const double a = fabs((double)v);
+        double p = a;
+        for (int r = 1; r < q; ++r) p = __dmul_rn(p, a);
+        acc += p;
+    }
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const float* __restrict__ grads)
+{
+    __shared__ double scratch[kThreads / 32];
+    const Tile tile = p.tiles[blockIdx.x];
+    const LayerDesc L = p.layers[tile.layer];
+    const int k = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float* __restrict__ g = grads + (int64_t)k * p.padded_elems + L.elem_off;
+
+    double acc = 0.0;
+    uint32_t maxbits = 0;
+    if (warp < tile.nblocks) {
+        const int64_t base = (int64_t)(tile.block0 + warp) * kBlockCoords + 4 * lane;
+        if (base - 4 * lane + kBlockCoords <= L.size) {
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                v[j] = __ldg(reinterpret_cast<const float4*>(g + base + 128 * j));
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                accumulate<kMode>(acc, maxbits, v[j].x, p.q);
+                accumulate<kMode>(acc, maxbits, v[j].y, p.q);
+                accumulate<kMode>(acc, maxbits, v[j].z, p.q);
+                accumulate<kMode>(acc, maxbits, v[j].w, p.q);
+            }
+        } else {
+            for (int j = 0; j < 8; ++j) {
+                const int64_t pos = base + 128 * j;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (pos + e < L.size) accumulate<kMode>(acc, maxbits, __ldg(g + pos + e), p.q);
+            }
+        }
+    }
+    if (kMode == 0)   // a non-finite maximum is handed on as NaN so that the final pass sees it
+        acc = maxbits >= 0x7f800000u ? __longlong_as_double(0x7ff8000000000000LL)
+                                     : (double)__uint_as_float(maxbits);
+    double r;
+    if (kMode == 0) {
+        // fmax drops NaNs: reduce a "bad" flag next to the maximum
+        const unsigned bad = __syncthreads_or(acc != acc);
+        r = block_reduce<true>(acc == acc ? acc : 0.0, scratch);
+        if (bad) r = __longlong_as_double(0x7ff8000000000000LL);
+    } else {
+        r = block_reduce<false>(acc, scratch);
+    }
+    if (threadIdx.x == 0) p.norm_partial[(int64_t)k * p.num_tiles + blockIdx.x] = r;
+}
+
+// One CTA per (layer, worker): adds the layer's tile partials (thread i takes partials
+// i, i+128, ... in order; then the fixed CTA tree), takes the root, rounds to fp32 and stores
+// the norm, its fp32 reciprocal and the status flags.
+__global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __restrict__ norms)
+{
+    __shared__ double scratch[4];
+    const int m = blockIdx.x, k = blockIdx.y;
+    const LayerDesc L = p.layers[m];
+    const double* part = p.norm_partial + (int64_t)k * p.num_tiles + L.first_tile;
+    double acc = 0.0;
+    int bad = 0;
+    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) {
+        const double v = part[i];
+        if (!(fabs(v) <= 1.7976931348623157e308)) bad = 1;
+        if (p.q == 0) acc = fmax(acc, v); else acc += v;
+    }
+    bad = __syncthreads_or(bad);
+    const double total = p.q == 0 ? block_reduce<true>(acc, scratch) : block_reduce<false>(acc, scratch);
+    if (threadIdx.x == 0) {
+        double n64;
+        if (p.q == 0 || p.q == 1) n64 = total;
+        else if (p.q == 2)        n64 = sqrt(total);
+        else                      n64 = pow(total, 1.0 / (double)p.q);
+        float n = (float)n64;
+        uint32_t st = 0;
+        if (bad || !(fabs(n64) <= 1.7976931348623157e308) || !(fabsf(n) <= 3.402823466e38f))
+            st = LQ_STATUS_NONFINITE;
+        else if (n < 1.17549435e-38f)
+            st = LQ_STATUS_ZERO_NORM;
+        if (st) n = 0.0f;
+        const int64_t o = (int64_t)k * p.num_layers + m;
+        norms[o] = n;
+        p.rnorm[o] = st ? 0.0f : __fdiv_rn(1.0f, n);
+        p.status[o] = st;
+    }
+}
+
+cudaError_t launch_norm(const PlanDev& p, const float* grads, float* norms, cudaStream_t s)
+{
+    if (p.num_tiles > 0) {
+        const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
+        if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads);
+        else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads);
+        else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads);
+        else               norm_partial_kernel<3><<<grid, kThreads, 0, s>>>(p, grads);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    norm_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p, norms);
+    return cudaGetLastError();
+}
+
+}  // namespace lq

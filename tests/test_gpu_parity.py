@@ -1,0 +1,260 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle on seeded inputs.
+
+Tolerances: packed signs and level indices bit-exact except coordinates within 1e-6 of a
+rounding threshold (fewer than 1e-6 of all coordinates); layer norms relative 1e-6; decoded
+and aggregated values relative 1e-6 (against the layer's largest magnitude); QODA iterates
+relative 1e-5.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import compare_messages, oracle_model, to_padded, to_unpadded
+
+pytestmark = pytest.mark.gpu
+SEED = 0x5EED0DA
+RAGGED = [0, 1, 31, 32, 33, 127, 128, 129, 1023, 1024, 1025, 8191, 8192, 8193, 20000, 3, 70001]
+
+
+@pytest.fixture(scope="module")
+def lqm():
+    import paper_2505_14371_b200 as pkg
+    pkg.load_library()
+    return pkg
+
+
+def _grads(plan, seed, scale=1.0):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    x = torch.randn((plan.num_workers, plan.padded_elems), generator=g, device="cuda") * scale
+    return x.contiguous()
+
+
+def _random_levels(rng, n):
+    inner = np.sort(rng.uniform(0.0, 1.0, n - 2) ** 3)
+    lv = np.concatenate([[0.0], inner, [1.0]]).astype(np.float32)
+    for j in range(1, n):                       # strictly increasing in fp32
+        if lv[j] <= lv[j - 1]:
+            lv[j] = np.nextafter(lv[j - 1], np.float32(2.0))
+    lv[-1] = 1.0
+    return lv
+
+
+def _close(a, b, rel, scale=None):
+    a = np.asarray(a, np.float64); b = np.asarray(b, np.float64)
+    s = np.max(np.abs(b)) if scale is None else scale
+    return np.max(np.abs(a - b), initial=0.0) <= rel * max(s, 1e-300)
+
+
+@pytest.mark.parametrize("q", [2, 0, 1, 3])
+def test_layer_norms(lqm, orc, q):
+    plan = lqm.Plan(RAGGED, 4, q, 3, SEED)
+    grads = _grads(plan, 1, 0.01)
+    norms = plan.empty_norms()
+    plan.lq_layer_norms(grads, norms)
+    g = to_unpadded(plan, grads)
+    off = np.concatenate([[0], np.cumsum(RAGGED)])
+    got = norms.cpu().numpy()
+    for k in range(3):
+        for m in range(len(RAGGED)):
+            ref, st = orc.layer_norm(g[k, off[m]:off[m + 1]], q)
+            assert abs(float(got[k, m]) - float(ref)) <= 1e-6 * float(ref), (k, m)
+    _, flags = plan.lq_get_statistics()
+    assert flags[:, 0].tolist() == [lqm.STATUS_ZERO_NORM] * 3 and int(flags[:, 1:].sum()) == 0
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_quantize_pack_all_widths_ragged(lqm, orc, bits):
+    rng = np.random.default_rng(bits)
+    plan = lqm.Plan(RAGGED, bits, 2, 2, SEED + bits)
+    if bits > 1:
+        for m in range(plan.num_layers):
+            if m % 2:
+                plan.lq_set_levels(m, _random_levels(rng, 1 << bits))
+    grads = _grads(plan, 10 + bits)
+    packed = plan.empty_packed(); norms = plan.empty_norms(); hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 5, packed, norms, hist=hist)
+    model = oracle_model(orc, plan)
+    ref = model.quantize(to_unpadded(plan, grads), 5, want_hist=True)
+    assert np.array_equal(norms.cpu().numpy()[:, :plan.num_layers], ref["norms"])
+    bad, stray = compare_messages(orc, plan, packed, ref)
+    assert bad == 0 and stray == 0
+    assert np.array_equal(hist.cpu().numpy().view(np.uint32), ref["hist"])
+    sq, _ = plan.lq_get_statistics()
+    assert _close(sq.numpy(), ref["sq_diff"], 1e-12)
+
+
+def test_config1_mlp_single_step(lqm, orc):
+    """4-layer MLP gradient set, K=4, 3-bit uniform levels: quantize -> decode-aggregate -> QODA."""
+    from paper_2505_14371_b200 import workloads as W
+    w = W.mlp_workload()
+    plan = lqm.Plan(w.layer_sizes, w.bits, w.q, w.num_workers, W.PHILOX_SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda")
+    packed = plan.empty_packed(); norms = plan.empty_norms()
+    gbar = torch.zeros(plan.padded_elems, device="cuda")
+    X1 = _grads(plan, 77)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    X = torch.empty_like(X1); g2 = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    plan.lq_quantize_pack(grads, 1, packed, norms)
+    plan.lq_decode_aggregate(packed, norms, gbar)
+    plan.qoda_step(packed, norms, X1, Y, Xh, X, g2)
+
+    model = oracle_model(orc, plan)
+    model.qoda_init(to_unpadded(plan, X1))
+    ref = model.quantize(to_unpadded(plan, grads), 1)
+    bad, stray = compare_messages(orc, plan, packed, ref)
+    total = w.num_coords * w.num_workers
+    assert stray == 0 and bad <= max(1, int(1e-6 * total)) and ref["near"] < 1e-5 * total
+    assert _close(norms.cpu().numpy(), ref["norms"], 1e-6)
+    gref = model.qoda_step()
+    off = np.concatenate([[0], np.cumsum(w.layer_sizes)])
+    if bad == 0:
+        for name, got, want in [("gbar", gbar, gref), ("gbar2", g2, gref), ("Y", Y, model.Y),
+                                ("X", X, model.X), ("Xhalf", Xh, model.Xhalf)]:
+            gg = to_unpadded(plan, got)
+            for m in range(plan.num_layers):
+                assert _close(gg[off[m]:off[m + 1]], want[off[m]:off[m + 1]], 1e-6), (name, m)
+    t, S, eta = plan.qoda_get_scalars()
+    assert t == 2 and abs(S - model.S) <= 1e-12 * model.S and eta == float(model.eta)
+
+
+def test_statistic_with_previous_message_and_level_change(lqm, orc):
+    rng = np.random.default_rng(4)
+    sizes = [5000, 33, 12345]
+    plan = lqm.Plan(sizes, [4, 3, 2], 2, 3, SEED)
+    model = oracle_model(orc, plan)
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    for step in range(1, 5):
+        if step == 3:                            # levels change between two messages
+            for m, b in enumerate(plan.bits):
+                lv = _random_levels(rng, 1 << b)
+                plan.lq_set_levels(m, lv); model.levels[m] = lv
+        grads = _grads(plan, 100 + step, 0.1)
+        cur, prv = pk[step % 2], pk[(step + 1) % 2]
+        plan.lq_quantize_pack(grads, step, cur, nm[step % 2],
+                              prev_packed=None if step == 1 else prv,
+                              prev_norms=None if step == 1 else nm[(step + 1) % 2])
+        ref = model.quantize(to_unpadded(plan, grads), step)
+        model.prev_decoded = ref["decoded"]
+        bad, stray = compare_messages(orc, plan, cur, ref)
+        assert bad == 0 and stray == 0
+        sq, _ = plan.lq_get_statistics()
+        assert _close(sq.numpy(), ref["sq_diff"], 1e-12), step
+
+
+@pytest.mark.parametrize("K", [1, 4, 11, 16])
+def test_decode_aggregate_worker_counts(lqm, orc, K):
+    sizes = [4100, 7, 1024, 2049]
+    plan = lqm.Plan(sizes, [4, 8, 1, 3], 0, K, SEED)
+    grads = _grads(plan, K)
+    packed = plan.empty_packed(); norms = plan.empty_norms()
+    gbar = torch.full((plan.padded_elems,), 7.0, device="cuda")
+    plan.lq_quantize_pack(grads, 9, packed, norms)
+    plan.lq_decode_aggregate(packed, norms, gbar)
+    model = oracle_model(orc, plan)
+    ref = model.quantize(to_unpadded(plan, grads), 9)
+    assert compare_messages(orc, plan, packed, ref) == (0, 0)
+    want = model.mean_decoded(ref["decoded"])
+    got = to_unpadded(plan, gbar)
+    assert np.array_equal(got, want)             # fixed summation order: bit-exact
+
+
+def test_nonfinite_and_zero_layers(lqm, orc):
+    sizes = [1500, 1500, 1500, 64]
+    plan = lqm.Plan(sizes, 4, 2, 2, SEED)
+    grads = _grads(plan, 3)
+    o = plan.elem_offsets
+    grads[0, o[1] + 5] = float("nan")
+    grads[1, o[2] + 1400] = float("inf")
+    grads[:, o[3]: o[3] + 64] = 0.0
+    packed = plan.empty_packed(); norms = plan.empty_norms(); gbar = torch.empty(plan.padded_elems, device="cuda")
+    plan.lq_quantize_pack(grads, 2, packed, norms)
+    plan.lq_decode_aggregate(packed, norms, gbar)
+    torch.cuda.synchronize()
+    _, flags = plan.lq_get_statistics()
+    assert flags.tolist() == [[0, lqm.STATUS_NONFINITE, 0, lqm.STATUS_ZERO_NORM],
+                              [0, 0, lqm.STATUS_NONFINITE, lqm.STATUS_ZERO_NORM]]
+    model = oracle_model(orc, plan)
+    ref = model.quantize(to_unpadded(plan, grads), 2)
+    assert ref["status"].tolist() == [[0, 2, 0, 1], [0, 0, 2, 1]]
+    assert compare_messages(orc, plan, packed, ref) == (0, 0)
+    assert np.array_equal(norms.cpu().numpy(), ref["norms"])
+    assert np.array_equal(to_unpadded(plan, gbar), model.mean_decoded(ref["decoded"]))
+    assert torch.isfinite(gbar[: o[3] + 64]).all()
+
+
+def test_fit_levels_parity(lqm, orc):
+    from paper_2505_14371_b200 import workloads as W
+    w = W.wgan_workload()
+    sizes = [s // 16 for s in w.layer_sizes]
+    w.layer_sizes = sizes
+    plan = lqm.Plan(sizes, [3, 4, 2, 8, 3, 4, 5, 3, 1], 2, 4, SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda", workers=4)
+    packed = plan.empty_packed(); norms = plan.empty_norms(); hist = plan.zero_hist()
+    model = oracle_model(orc, plan)               # holds the levels before the fit
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels(hist, norms, 4)
+    h = hist.cpu().numpy().view(np.uint32); n = norms.cpu().numpy()
+    for m, b in enumerate(plan.bits):
+        got = np.array(plan.lq_get_levels(m))
+        want = orc.fit_levels(h[:, m, :], n[:, m], sizes[m], 1 << b)
+        if want is None:
+            want = model.levels[m]
+        assert np.allclose(got, want, rtol=1e-6, atol=0), m
+        assert got[0] == 0 and got[-1] == 1 and np.all(np.diff(got) > 0)
+    # the fitted levels are used by the next message, and the previous one still decodes with the old ones
+    packed2 = plan.empty_packed(); norms2 = plan.empty_norms()
+    plan.lq_quantize_pack(grads, 2, packed2, norms2, prev_packed=packed, prev_norms=norms)
+    ref1 = model.quantize(to_unpadded(plan, grads), 1)
+    model.prev_decoded = ref1["decoded"]
+    for m in range(plan.num_layers):
+        model.levels[m] = np.array(plan.lq_get_levels(m), np.float32)
+    ref2 = model.quantize(to_unpadded(plan, grads), 2)
+    assert compare_messages(orc, plan, packed2, ref2) == (0, 0)
+    sq, _ = plan.lq_get_statistics()
+    assert _close(sq.numpy(), ref2["sq_diff"], 1e-12)
+
+
+def test_qoda_multi_step_small(lqm, orc):
+    """20 iterations with random 'gradients' that depend on nothing: state parity every step."""
+    sizes = [3000, 100, 2048]
+    plan = lqm.Plan(sizes, 4, 2, 4, SEED)
+    model = oracle_model(orc, plan)
+    X1 = _grads(plan, 5)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    model.qoda_init(to_unpadded(plan, X1))
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    for t in range(1, 21):
+        grads = _grads(plan, 1000 + t, 1.0 / t)
+        c, p = t % 2, (t + 1) % 2
+        plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=None if t == 1 else pk[p],
+                              prev_norms=None if t == 1 else nm[p])
+        plan.qoda_step(pk[c], nm[c], X1, Y, Xh)
+        ref = model.quantize(to_unpadded(plan, grads), t)
+        assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+        model.qoda_step()
+        tt, S, eta = plan.qoda_get_scalars()
+        assert tt == t + 1 and abs(S - model.S) <= 1e-12 * model.S and eta == float(model.eta)
+        assert _close(to_unpadded(plan, Y), model.Y, 1e-6) and _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
+
+
+def test_argument_errors(lqm):
+    with pytest.raises(lqm.LqError):
+        lqm.Plan([10], 9, 2, 1, 0)
+    with pytest.raises(lqm.LqError):
+        lqm.Plan([10], 4, 17, 1, 0)
+    with pytest.raises(lqm.LqError):
+        lqm.Plan([10], 4, 2, 0, 0)
+    plan = lqm.Plan([10], 2, 2, 1, 0)
+    with pytest.raises(lqm.LqError):
+        plan.lq_set_levels(0, [0.0, 0.5, 0.5, 1.0])
+    with pytest.raises(lqm.LqError):
+        plan.lq_set_levels(0, [0.0, 0.5, 1.0])
+    with pytest.raises(lqm.LqError):
+        plan.lq_set_levels(0, [0.1, 0.5, 0.7, 1.0])
+    X = torch.zeros(plan.padded_elems, device="cuda")
+    with pytest.raises(lqm.LqError):              # qoda_step before qoda_init
+        plan.qoda_step(plan.empty_packed(), plan.empty_norms(), X, X.clone(), X.clone())
+    empty = lqm.Plan([], 4, 2, 2, 0)
+    assert empty.packed_words == 0
