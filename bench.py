@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of the QODA hot path on B200: one step = lq_quantize_pack (norm + stochastic
+rounding + packing + step-size statistic) followed by qoda_step (fused decode + aggregate +
+update) over one Transformer-XL-shaped synthetic gradient set for K = 8 simulated workers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+Prints ONE JSON line.  `value` is GB/s of fp32 input (4*K*D bytes per step) with the inputs
+resident in HBM; `e2e` is the same with the gradients copied from pinned host memory and the
+new iterate copied back inside the timed region.  With --impl reference the CPU oracle is timed
+on a bounded sample instead.  With N > 1 (launched by torch.distributed.run) every rank runs an
+independent replica of the workload: the method does not shard inside one node's GPU, so there
+is no collective on the data path, only the barrier and the max-over-ranks of the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "quantize+pack and decode+aggregate+QODA GB/s (fp32 in)"
+
+
+# ------------------------------------------------------------------------------ workloads
+def pick_workload(name: str):
+    from paper_2505_14371_b200 import workloads as W
+    if name == "transformer_xl":
+        return W.transformer_xl_workload()
+    if name == "wgan":
+        return W.wgan_workload()
+    if name == "mlp":
+        return W.mlp_workload()
+    if name == "transformer_xl_small":
+        return W.transformer_xl_workload(num_blocks=2, vocab=8192)
+    raise SystemExit(f"unknown workload {name}")
+
+
+# --------------------------------------------------------------------------- clock sampler
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15] or [r for _, r in self.rows[-3:]]
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# -------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample_workload():
+    """Bounded sample of the Transformer-XL-shaped workload for the CPU oracle: 8192 embedding
+    rows and one transformer block, all 8 workers, same value recipe."""
+    from paper_2505_14371_b200 import workloads as W
+    return W.transformer_xl_workload(num_blocks=1, vocab=8192)
+
+
+def time_oracle(steps: int, warmup: int) -> dict:
+    """Times the oracle (as it stands, single-threaded C behind ctypes) on the sample."""
+    import numpy as np
+    import torch
+    from oracle import oracle as orc
+    from paper_2505_14371_b200 import workloads as W
+    orc.build()
+    w = oracle_sample_workload()
+    offs = np.concatenate([[0], np.cumsum(w.layer_sizes)]).astype(np.int64)
+    D = int(offs[-1])
+    grads = W.make_gradients(w, [int(x) for x in offs[:-1]], D, "cpu").numpy()
+    model = orc.OracleModel(w.layer_sizes, [w.bits] * w.num_layers, w.q, w.num_workers, W.PHILOX_SEED)
+    g = torch.Generator(device="cpu").manual_seed(W.SEED_BASE + 99)
+    model.qoda_init(torch.randn(D, generator=g).numpy())
+    times = []
+    for s in range(warmup + steps):
+        t0 = time.perf_counter()
+        model.quantize(grads, s + 1)
+        model.qoda_step()
+        t1 = time.perf_counter()
+        if s >= warmup:
+            times.append(t1 - t0)
+    sec = sum(times) / len(times)
+    return {"value": 4.0 * w.num_workers * D / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"transformer_xl shapes cut to 8192 embedding rows + 1 block "
+                      f"({D} coords x K={w.num_workers}), {len(times)} step(s), {sec:.2f} s/step",
+            "ms_per_step": sec * 1e3}
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps, warmup = max(1, min(args.steps, 3)), min(args.warmup, 1)
+    r = time_oracle(steps, warmup)
+    w = pick_workload(args.workload)
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "transformer_xl_shaped", "num_workers": w.num_workers, "bits": w.bits,
+                       "q": w.q, "note": "CPU oracle on a bounded sample of this workload"},
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------- GPU leg
+def aggregate_over_ranks(local_ms: float, world: int, device=None, backend_reduce=None) -> float:
+    """Max over ranks of the per-rank step time (host logic shared with the CPU gloo test)."""
+    if world == 1:
+        return local_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, max_ms: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time (weak scaling)."""
+    return units_per_rank * world / (max_ms * 1e-3)
+
+
+def run_gpu(args) -> None:
+    import torch
+    import torch.distributed as dist
+    import paper_2505_14371_b200 as pkg
+    from paper_2505_14371_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    pkg.load_library()
+
+    w = pick_workload(args.workload)
+    K, D = w.num_workers, w.num_coords
+    plan = pkg.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, dev)
+    packed = [plan.empty_packed(dev), plan.empty_packed(dev)]
+    norms = [plan.empty_norms(dev), plan.empty_norms(dev)]
+    g = torch.Generator(device=dev).manual_seed(W.SEED_BASE + 99)
+    X1 = torch.randn(plan.padded_elems, generator=g, device=dev)
+    Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+
+    state = {"t": 0}
+
+    def step():
+        state["t"] += 1
+        t = state["t"]
+        c, p = t % 2, (t + 1) % 2
+        plan.lq_quantize_pack(grads, t, packed[c], norms[c],
+                              prev_packed=None if t == 1 else packed[p],
+                              prev_norms=None if t == 1 else norms[p])
+        plan.qoda_step(packed[c], norms[c], X1, Y, Xh)
+
+    # adaptive levels: one histogram + fit before the steady state (Algorithm 1 lines 2-7)
+    hist = plan.zero_hist(dev)
+    state["t"] += 1
+    plan.lq_quantize_pack(grads, 1, packed[1], norms[1], hist=hist)
+    plan.lq_fit_levels(hist, norms[1], K)
+    plan.qoda_step(packed[1], norms[1], X1, Y, Xh)
+    del hist
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ----------------------------------------------------------
+    sampler = ClockSampler(local)
+    plan.lq_profile_enable(True); plan.lq_profile_read()
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    local_ms = e0.elapsed_time(e1) / args.steps
+    prof = plan.lq_profile_read()
+    plan.lq_profile_enable(False)
+    ms = aggregate_over_ranks(local_ms, world, dev)
+
+    # ---- end to end: pinned host gradients in, new iterate out ------------------------------
+    e2e = None
+    try:
+        host_grads = torch.empty(grads.shape, dtype=torch.float32, pin_memory=True)
+        host_grads.copy_(grads)
+        host_out = torch.empty(Xh.shape, dtype=torch.float32, pin_memory=True)
+        e2e_steps = max(1, min(args.steps, 5))
+
+        def e2e_step():
+            grads.copy_(host_grads, non_blocking=True)
+            step()
+            host_out.copy_(Xh, non_blocking=True)
+
+        e2e_step(); barrier()
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = aggregate_over_ranks(e0.elapsed_time(e1) / e2e_steps, world, dev)
+        e2e = {"value": whole_job_value(4.0 * K * D / 1e9, world, e2e_ms), "unit": "GB/s",
+               "h2d_bytes_per_step": host_grads.numel() * 4, "d2h_bytes_per_step": host_out.numel() * 4,
+               "ms_per_step": e2e_ms}
+        del host_grads, host_out
+    except RuntimeError as exc:      # pinned allocation can fail on a small host
+        e2e = {"value": None, "unit": "GB/s", "error": str(exc)[:200]}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel --------------------------------------------------
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = 6650.0, "fallback"
+    c = (w.bits + 1) / 8.0
+    # algorithmic bytes per launch: what the method itself must move, per kernel
+    alg = {"norm_partial": 4.0 * K * D, "quantize_pack": (4.0 + 2 * c) * K * D, "decode": (K * c + 16.0) * D}
+    kern = {}
+    for name, (tot, cnt) in prof.items():
+        if cnt:
+            avg = tot / cnt
+            kern[name] = {"avg_ms": avg, "launches_per_step": cnt / args.steps}
+            if name in alg:
+                kern[name]["gbs"] = alg[name] / (avg * 1e-3) / 1e9
+                kern[name]["frac"] = kern[name]["gbs"] / peak
+    dominant = max((n for n in kern if n in alg), key=lambda n: kern[n]["avg_ms"] * kern[n]["launches_per_step"])
+    traffic_path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    traffic = None
+    if os.path.exists(traffic_path):
+        traffic = json.load(open(traffic_path)).get(args.workload, {}).get(dominant)
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": kern[dominant]["gbs"], "peak": peak,
+                "peak_source": peak_src, "unit": "GB/s", "frac": kern[dominant]["frac"], "traffic": traffic,
+                "algorithmic_bytes_per_launch": alg[dominant], "kernels": kern}
+    qp_ms = sum(kern[n]["avg_ms"] for n in ("norm_partial", "norm_finalize", "quantize_pack", "stat_finalize") if n in kern)
+    st_ms = sum(kern[n]["avg_ms"] for n in ("qoda_scalars", "decode") if n in kern)
+    calls = {"lq_quantize_pack": {"ms": qp_ms, "fp32_in_gbs": 4.0 * K * D / qp_ms / 1e6,
+                                  "algorithmic_gbs": (8.0 + 2 * c) * K * D / qp_ms / 1e6,
+                                  "frac_of_peak": (8.0 + 2 * c) * K * D / qp_ms / 1e6 / peak},
+             "qoda_step": {"ms": st_ms, "fp32_equiv_gbs": 4.0 * K * D / st_ms / 1e6,
+                           "algorithmic_gbs": (K * c + 16.0) * D / st_ms / 1e6,
+                           "frac_of_peak": (K * c + 16.0) * D / st_ms / 1e6 / peak}}
+
+    cpu = time_oracle(3, 0) if world == 1 and not args.no_cpu_baseline else None
+    launches = int(sum(cnt for _, cnt in prof.values()))
+    line = {"metric": METRIC, "value": whole_job_value(4.0 * K * D / 1e9, world, ms), "unit": "GB/s",
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}_shaped", "coords": D, "layers": w.num_layers, "num_workers": K,
+                       "bits": w.bits, "q": w.q, "levels": "adaptive (fitted once before timing)",
+                       "l2": "inputs (%.2f GB) exceed L2" % (4.0 * K * D / 1e9),
+                       "multi_gpu": "replicas only"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "calls": calls}
+    if cpu:
+        line["cpu_baseline"] = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="transformer_xl")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

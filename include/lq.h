@@ -13,7 +13,7 @@
  *    take a stream only enqueue work on it and return; they do not synchronise unless
  *    stated.  Calls on one plan must be issued in stream order by the caller.
  *  - Argument errors are reported synchronously.  Data problems (NaN/Inf input, zero
- *    norm) never fault: they set per-(worker, layer) status flags, see lq_get_status.
+ *    norm) never fault: they set per-(worker, layer) status flags, see lq_get_statistics.
  *
  * Data layout
  *  - A plan is a ragged list of L layers with sizes d_m, code widths b_m (n_m = 2^b_m levels
@@ -23,11 +23,12 @@
  *    and its d_m values are contiguous.  grads is [K][D_pad], row-major.  Elements between
  *    layers are padding: never interpreted on input, may be overwritten on output.
  *  - A worker's message is W = lq_plan_packed_words() 32-bit words; packed is [K][W].
+ *    Every coordinate becomes one symbol of b+1 bits, symbol = sign * 2^b + level index.
  *    Layer m starts at word_off_m and is cut into blocks of 1024 coordinates (the last one
  *    zero-padded).  A block is (b+1) planes of 32 words.  Coordinate c of a block belongs to
- *    lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane.  Plane 0 holds the sign
- *    bits (bit p of word `lane`); planes 1..b hold, per lane, the 32 level indices as one
- *    little-endian string of 32*b bits with index p at bit offset p*b (word `plane*32+lane`).
+ *    lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane.  The 32 symbols of a lane
+ *    form one little-endian string of 32*(b+1) bits with symbol p at bit offset p*(b+1); bit t
+ *    of that string is bit t%32 of word (t/32)*32 + lane of the block.
  *    The norms travel separately as fp32: norms is [K][L].
  *    (Section 3.2 of the paper fixes the content of a message: a 32-bit float norm, one sign
  *    bit and one integer code per coordinate; the physical arrangement is this library's.)
@@ -76,7 +77,8 @@ int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, in
                        int32_t* num_levels);
 
 /* Level sequence of one layer (Section 3.1: 0 = l_0 < l_1 < ... < l_{n-1} = 1, n = 2^b).
- * host_levels [n] host.  set: validates (n must equal 2^b, strictly increasing, ends 0 and 1)
+ * host_levels [n] host.  set: validates (n must equal 2^b, increasing by at least 2^-100 per
+ * step, ends 0 and 1)
  * and stages the sequence; it is used from the next lq_quantize_pack on.  get: returns the
  * staged sequence (the most recent of set / fit).  Both synchronise the device. */
 int lq_set_levels(lq_plan* plan, int32_t layer, const float* host_levels, int32_t n);
@@ -146,6 +148,23 @@ int qoda_get_scalars(const lq_plan* plan, int64_t* t, double* S, double* eta);
  * (host_sq_diff [K][L] doubles) and status flags (host_flags [K][L], LQ_STATUS_*) of the
  * last norm computation.  Either may be NULL.  Synchronises. */
 int lq_get_statistics(const lq_plan* plan, double* host_sq_diff, uint32_t* host_flags);
+
+/* Measurement aid (no counterpart in the paper).  While enabled, every kernel the library
+ * launches for this plan is bracketed by two CUDA events on the caller's stream.
+ * lq_profile_read synchronises the device, returns per kernel the summed device time in
+ * milliseconds and the number of launches since the last read (arrays of LQ_NUM_KERNELS,
+ * indexed by LQ_KERNEL_*), and clears the record.  At most 65536 launches are recorded
+ * between two reads. */
+#define LQ_KERNEL_NORM_PARTIAL   0
+#define LQ_KERNEL_NORM_FINALIZE  1
+#define LQ_KERNEL_QUANTIZE_PACK  2
+#define LQ_KERNEL_STAT_FINALIZE  3
+#define LQ_KERNEL_QODA_SCALARS   4
+#define LQ_KERNEL_DECODE         5
+#define LQ_KERNEL_FIT            6
+#define LQ_NUM_KERNELS           7
+int lq_profile_enable(lq_plan* plan, int32_t enable);
+int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches);
 
 const char* lq_error_string(int code);
 const char* lq_last_error(void);

@@ -147,11 +147,12 @@ double orc_round_up_probability(double u, const float* level, int n, int* tau_ou
  * Fixed-width message layout (Section 3.2: a 32-bit float norm, one sign bit and one
  * integer code per coordinate; Section 7.1 footnote: no entropy code on top).
  * The physical layout is this build's:
- *   a layer of d coordinates with b-bit codes is cut into blocks of 1024 coordinates
- *   (the last one zero-padded); a block is (b+1) planes of 32 words; coordinate c of a
- *   block belongs to lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane;
- *   plane 0 holds the signs (bit p of the lane's word); planes 1..b hold, per lane, the
- *   32 codes as one little-endian string of 32*b bits with code p at bit offset p*b.
+ *   every coordinate becomes one symbol of b+1 bits, symbol = sign * 2^b + idx;
+ *   a layer of d coordinates is cut into blocks of 1024 coordinates (the last one
+ *   zero-padded); a block is (b+1) planes of 32 words; coordinate c of a block belongs to
+ *   lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane; the 32 symbols of a
+ *   lane form one little-endian string of 32*(b+1) bits with symbol p at bit offset
+ *   p*(b+1); bit t of that string is bit t%32 of word (t/32)*32 + lane of the block.
  * ---------------------------------------------------------------------------------- */
 int64_t orc_packed_words(int64_t d, int b)
 {
@@ -173,11 +174,11 @@ void orc_pack_layer(const uint8_t* idx, const uint8_t* sign, int64_t d, int b, u
     for (int64_t i = 0; i < d; ++i) {
         int64_t base; int lane, p;
         locate(i, b, &base, &lane, &p);
-        if (sign[i]) words[base + lane] |= (uint32_t)1 << p;
-        for (int bit = 0; bit < b; ++bit) {
-            if ((idx[i] >> bit) & 1) {
-                int pos = p * b + bit;               /* position in the 32*b-bit string */
-                words[base + (int64_t)(1 + pos / 32) * 32 + lane] |= (uint32_t)1 << (pos % 32);
+        unsigned symbol = ((unsigned)(sign[i] ? 1 : 0) << b) | idx[i];
+        for (int bit = 0; bit <= b; ++bit) {
+            if ((symbol >> bit) & 1u) {
+                int t = p * (b + 1) + bit;           /* position in the lane's bit string */
+                words[base + (int64_t)(t / 32) * 32 + lane] |= (uint32_t)1 << (t % 32);
             }
         }
     }
@@ -188,13 +189,13 @@ void orc_unpack_layer(const uint32_t* words, int64_t d, int b, uint8_t* idx, uin
     for (int64_t i = 0; i < d; ++i) {
         int64_t base; int lane, p;
         locate(i, b, &base, &lane, &p);
-        sign[i] = (uint8_t)((words[base + lane] >> p) & 1u);
-        unsigned code = 0;
-        for (int bit = 0; bit < b; ++bit) {
-            int pos = p * b + bit;
-            code |= ((words[base + (int64_t)(1 + pos / 32) * 32 + lane] >> (pos % 32)) & 1u) << bit;
+        unsigned symbol = 0;
+        for (int bit = 0; bit <= b; ++bit) {
+            int t = p * (b + 1) + bit;
+            symbol |= ((words[base + (int64_t)(t / 32) * 32 + lane] >> (t % 32)) & 1u) << bit;
         }
-        idx[i] = (uint8_t)code;
+        idx[i] = (uint8_t)(symbol & ((1u << b) - 1u));
+        sign[i] = (uint8_t)(symbol >> b);
     }
 }
 
@@ -241,7 +242,8 @@ void orc_histogram_layer(const float* v, int64_t d, float norm, uint32_t* hist)
  *     a < c, i.e. F~(l) = F~(c) - int_a^c (u-a)/(c-a) dF~(u)  (the first-order condition
  *     int_a^l (u-a) dF~ = int_l^c (c-u) dF~), odd levels first, then even levels;
  *   up to 100 sweeps, stopping when no level moved by more than 1e-13 relative;
- *   round to fp32 and force strict monotonicity by single-ulp steps.
+ *   round to fp32 and force strict monotonicity: each level at least one ulp and at least
+ *   2^-40 above the one before, and at least one ulp below the one after.
  * Returns 1 if levels were written, 0 if there was no usable mass (levels untouched).
  * hist is [Z][stride] counts, norms are the Z vectors' fp32 norms, d the layer size.
  * ---------------------------------------------------------------------------------- */
@@ -344,6 +346,8 @@ int orc_fit_levels(const uint32_t* hist, int64_t stride, const float* norms, int
     for (int j = 1; j <= n - 2; ++j) {
         float f = (float)l[j];
         float floor_ = nextafterf(level_out[j - 1], 2.0f);
+        float gap_ = level_out[j - 1] + 9.094947017729282e-13f;     /* previous level + 2^-40 */
+        if (gap_ > floor_) floor_ = gap_;
         level_out[j] = f > floor_ ? f : floor_;
     }
     for (int j = n - 2; j >= 1; --j) {

@@ -24,7 +24,10 @@ STATUS_NONFINITE = 2
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "lq_get_statistics", "lq_error_string", "lq_last_error"]
+           "qoda_get_scalars", "lq_get_statistics", "lq_profile_enable", "lq_profile_read",
+           "lq_error_string", "lq_last_error"]
+KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
+                "decode", "fit"]
 
 
 class LqError(RuntimeError):
@@ -59,6 +62,8 @@ def load_library() -> C.CDLL:
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
+    L.lq_profile_enable.argtypes = [vp, i32]
+    L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     L.lq_error_string.argtypes = [C.c_int]; L.lq_error_string.restype = C.c_char_p
     L.lq_last_error.argtypes = []; L.lq_last_error.restype = C.c_char_p
     for name in EXPORTS:
@@ -177,6 +182,16 @@ class Plan:
         _check(load_library().lq_get_statistics(self._h, sq, fl))
         return (torch.tensor(list(sq), dtype=torch.float64).view(K, Ln)[:, : self.num_layers],
                 torch.tensor(list(fl), dtype=torch.int64).view(K, Ln)[:, : self.num_layers])
+
+    def lq_profile_enable(self, enable: bool) -> None:
+        _check(load_library().lq_profile_enable(self._h, 1 if enable else 0))
+
+    def lq_profile_read(self):
+        """Returns {kernel name: (total ms, launches)} since the last read."""
+        n = len(KERNEL_NAMES)
+        ms = (C.c_double * n)(); cnt = (C.c_int64 * n)()
+        _check(load_library().lq_profile_read(self._h, ms, cnt))
+        return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n)}
 
     # ---- allocation helpers (device memory only; no arithmetic) ----------------------------
     def empty_packed(self, device="cuda") -> torch.Tensor:

@@ -48,11 +48,17 @@ struct lq_plan {
     Tile* d_tiles = nullptr;
     float* d_levels_stage = nullptr;
     float* d_levels_enc[2] = {nullptr, nullptr};
+    SearchTables search{};         // derived from d_levels_enc[cur]
     int cur = 0, prev = 0;
     bool stage_dirty = false;
     bool have_message = false;
     bool qoda_ready = false;
     bool stat_pending = false;
+    // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
+    struct ProfRec { int id; cudaEvent_t a, b; };
+    bool profiling = false;
+    std::vector<ProfRec> prof_recs;
+    std::vector<cudaEvent_t> prof_pool;
 };
 
 namespace {
@@ -62,9 +68,34 @@ void free_plan(lq_plan* p)
     if (!p) return;
     cudaFree(p->d_layers); cudaFree(p->d_tiles);
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
+    cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
     cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars);
+    for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
+}
+
+cudaEvent_t prof_event(lq_plan* p)
+{
+    cudaEvent_t e = nullptr;
+    if (!p->prof_pool.empty()) { e = p->prof_pool.back(); p->prof_pool.pop_back(); }
+    else if (cudaEventCreate(&e) != cudaSuccess) e = nullptr;
+    return e;
+}
+
+// Runs one launcher; when profiling is on, brackets it with two events on the same stream.
+template <typename F>
+cudaError_t timed(lq_plan* p, int id, cudaStream_t s, F&& launch)
+{
+    if (!p->profiling || p->prof_recs.size() >= 65536) return launch();
+    cudaEvent_t a = prof_event(p), b = prof_event(p);
+    if (!a || !b) return launch();
+    cudaEventRecord(a, s);
+    const cudaError_t e = launch();
+    cudaEventRecord(b, s);
+    p->prof_recs.push_back({id, a, b});
+    return e;
 }
 
 template <typename T>
@@ -153,6 +184,10 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_stage, lev);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[0], lev);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[1], lev);
+    const size_t nl = (size_t)(num_layers ? num_layers : 1);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.lut, nl * kLutStride);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.ld, nl * kMaxLevels);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.fast, nl);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.stat_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
@@ -184,6 +219,12 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
         return fail(code, "plan setup: %s", cudaGetErrorString(e));
     }
     d.layers = p->d_layers; d.tiles = p->d_tiles;
+    e = launch_build_search(d, p->d_levels_enc[0], p->search, nullptr);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        free_plan(p);
+        return fail(LQ_ECUDA, "plan setup: %s", cudaGetErrorString(e));
+    }
     *out = p;
     return LQ_OK;
 }
@@ -246,7 +287,10 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
 {
     if (!plan || !grads || !norms) return fail(LQ_EINVAL, "NULL argument");
     if (plan->dev.num_layers == 0) return LQ_OK;
-    LQ_CUDA(launch_norm(plan->dev, grads, norms, (cudaStream_t)stream));
+    cudaStream_t s = (cudaStream_t)stream;
+    const PlanDev& d = plan->dev;
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
     return LQ_OK;
 }
 
@@ -267,12 +311,20 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
         plan->prev = plan->cur;
         plan->cur = next;
         plan->stage_dirty = false;
+        LQ_CUDA(launch_build_search(plan->dev, plan->d_levels_enc[next], plan->search, s));
     } else {
         plan->prev = plan->cur;
     }
-    LQ_CUDA(launch_norm(plan->dev, grads, norms, s));
-    LQ_CUDA(launch_quantize(plan->dev, grads, step, packed, norms, hist, prev_packed, prev_norms,
-                            plan->d_levels_enc[plan->cur], plan->d_levels_enc[plan->prev], s));
+    const PlanDev& d = plan->dev;
+    const float* lc = plan->d_levels_enc[plan->cur];
+    const float* lp = plan->d_levels_enc[plan->prev];
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_QUANTIZE_PACK, s, [&] {
+        return launch_quantize(d, grads, step, packed, norms, hist, prev_packed, prev_norms, lc, lp,
+                               plan->search, s);
+    }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_stat_finalize(d, s); }));
     plan->have_message = true;
     plan->stat_pending = true;
     return LQ_OK;
@@ -283,7 +335,10 @@ int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32
     if (!plan || !hist || !norms) return fail(LQ_EINVAL, "NULL argument");
     if (num_samples < 1 || num_samples > LQ_MAX_WORKERS)
         return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
-    LQ_CUDA(launch_fit(plan->dev, hist, norms, num_samples, plan->d_levels_stage, (cudaStream_t)stream));
+    cudaStream_t s = (cudaStream_t)stream;
+    LQ_CUDA(timed(plan, LQ_KERNEL_FIT, s, [&] {
+        return launch_fit(plan->dev, hist, norms, num_samples, plan->d_levels_stage, s);
+    }));
     plan->stage_dirty = true;
     return LQ_OK;
 }
@@ -291,8 +346,12 @@ int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32
 int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float* norms, float* gbar, void* stream)
 {
     if (!plan || !packed || !norms || !gbar) return fail(LQ_EINVAL, "NULL argument");
-    LQ_CUDA(launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], nullptr, nullptr, nullptr,
-                          nullptr, gbar, false, (cudaStream_t)stream));
+    cudaStream_t s = (cudaStream_t)stream;
+    lq_plan* mp = const_cast<lq_plan*>(plan);      // the profiler's bookkeeping is not plan state
+    LQ_CUDA(timed(mp, LQ_KERNEL_DECODE, s, [&] {
+        return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], nullptr, nullptr,
+                             nullptr, nullptr, gbar, false, s);
+    }));
     return LQ_OK;
 }
 
@@ -312,9 +371,11 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
     if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
     if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
     cudaStream_t s = (cudaStream_t)stream;
-    LQ_CUDA(launch_qoda_scalars(plan->dev, s));
-    LQ_CUDA(launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
-                          gbar_opt, true, s));
+    LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_qoda_scalars(plan->dev, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
+        return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
+                             gbar_opt, true, s);
+    }));
     plan->stat_pending = false;
     return LQ_OK;
 }
@@ -340,6 +401,31 @@ int lq_get_statistics(const lq_plan* plan, double* host_sq_diff, uint32_t* host_
         LQ_CUDA(cudaMemcpy(host_sq_diff, plan->dev.sq_diff, KL * sizeof(double), cudaMemcpyDeviceToHost));
     if (host_flags && KL)
         LQ_CUDA(cudaMemcpy(host_flags, plan->dev.status, KL * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return LQ_OK;
+}
+
+int lq_profile_enable(lq_plan* plan, int32_t enable)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    plan->profiling = enable != 0;
+    return LQ_OK;
+}
+
+int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches)
+{
+    if (!plan || !total_ms || !launches) return fail(LQ_EINVAL, "NULL argument");
+    for (int i = 0; i < LQ_NUM_KERNELS; ++i) { total_ms[i] = 0.0; launches[i] = 0; }
+    LQ_CUDA(cudaDeviceSynchronize());
+    for (auto& r : plan->prof_recs) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess && r.id >= 0 && r.id < LQ_NUM_KERNELS) {
+            total_ms[r.id] += (double)ms;
+            launches[r.id] += 1;
+        }
+        plan->prof_pool.push_back(r.a);
+        plan->prof_pool.push_back(r.b);
+    }
+    plan->prof_recs.clear();
     return LQ_OK;
 }
 

@@ -1,9 +1,9 @@
 // DECODE + aggregate of the K workers' messages, alone or fused with the optimistic dual averaging
 // update (Algorithm 1 lines 15-18 and line 10 of the next iteration; Eq. ODA; Eq. general_stepsize).
 //
-// One CTA per tile (up to 8 blocks of 1024 coordinates of one layer), one warp per block.  A lane
+// One CTA per tile (up to 32 blocks of 1024 coordinates of one layer, taken round-robin by 8 warps).  A lane
 // owns the same 32 coordinates it owned at encode time, so it reads (b+1) words per worker with
-// 128-byte coalesced warp loads, looks the decoded values up in a per-(worker, layer) table in shared
+// 128-byte coalesced warp loads, looks the signed decoded values up by symbol in a per-(worker, layer) table in shared
 // memory, sums them in worker order in registers, and finishes with float4 reads of Y and X_1 and
 // float4 writes of Y and X_{t+3/2}.  Every packed word and every state element is touched once.
 #include "lq_internal.cuh"
@@ -12,28 +12,31 @@ namespace lq {
 
 constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
 
-template <int B>
-__device__ __forceinline__ uint32_t code_at(const uint32_t (&cw)[B], int p)
+// symbol p (pre-scaled by 4) of a lane's string of 32 symbols of C bits, held in C words
+template <int C>
+__device__ __forceinline__ uint32_t symbol4_at(const uint32_t (&w)[C], int p)
 {
-    const int off = p * B, w = off >> 5, s = off & 31;
-    uint32_t v = cw[w] >> s;
-    if (s + B > 32) v |= cw[w + 1] << (32 - s);
-    return v & ((1u << B) - 1u);
+    const int off = p * C, i = off >> 5, s = off & 31;
+    constexpr uint32_t mask4 = ((1u << C) - 1u) << 2;
+    uint32_t v;
+    if (s + C <= 32) v = s >= 2 ? (w[i] >> (s - 2)) : (w[i] << (2 - s));
+    else             v = __funnelshift_r(w[i], w[i + 1], s - 2);      // s >= 2 whenever a symbol straddles
+    return v & mask4;
 }
 
+// Adds one worker's decoded block into acc.  `table` holds N * l_j for j < n and -N * l_j after.
 template <int B>
 __device__ __forceinline__ void decode_accumulate(float (&acc)[32], const uint32_t* __restrict__ words,
                                                   const float* __restrict__ table)
 {
-    const uint32_t signw = words[0];
-    uint32_t cw[B];
+    constexpr int C = B + 1;
+    uint32_t w[C];
 #pragma unroll
-    for (int w = 0; w < B; ++w) cw[w] = words[(w + 1) * 32];
+    for (int i = 0; i < C; ++i) w[i] = __ldcs(words + i * 32);
+    const char* tb = reinterpret_cast<const char*>(table);
 #pragma unroll
-    for (int p = 0; p < 32; ++p) {
-        const uint32_t mag = __float_as_uint(table[code_at<B>(cw, p)]);
-        acc[p] += __uint_as_float(mag ^ ((signw >> p) << 31));
-    }
+    for (int p = 0; p < 32; ++p)
+        acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w, p));
 }
 
 struct DecodeArgs {
@@ -50,32 +53,45 @@ struct DecodeArgs {
 // Any worker count: the accumulators live across chunks of kWorkerChunk workers.
 template <int B, bool kQoda>
 __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
-                                                     int64_t blk, bool active, const DecodeArgs& a,
-                                                     float (*table)[kMaxLevels], float eta)
+                                                     const Tile& tile, const DecodeArgs& a,
+                                                     float (*table)[2 * kMaxLevels], float eta)
 {
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int K = p.num_workers;
+    const float invK = __fdiv_rn(1.0f, (float)K);
+    // each warp takes the tile's blocks round-robin; all warps run the same number of rounds so
+    // that the table refills (CTA-wide barriers) stay aligned
+    for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
+    const bool active = b0 + warp < tile.nblocks;
+    const int64_t blk = tile.block0 + b0 + warp;
     const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
     float acc[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
 
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
+        if (K <= kWorkerChunk && b0 > 0) {          // one chunk only: the table is already in place
+            if (active)
+                for (int kk = 0; kk < K; ++kk)
+                    decode_accumulate<B>(acc, a.packed + (int64_t)kk * p.packed_words + woff, table[kk]);
+            break;
+        }
         const int kc = min(kWorkerChunk, K - k0);
         __syncthreads();
         for (int i = threadIdx.x; i < kc * L.nlevels; i += blockDim.x) {
             const int kk = i / L.nlevels, j = i - kk * L.nlevels;
-            table[kk][j] = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
-                                     a.levels[(int64_t)layer * kLevelStride + j]);
+            const float mag = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
+                                        a.levels[(int64_t)layer * kLevelStride + j]);
+            table[kk][j] = mag;
+            table[kk][L.nlevels + j] = -mag;
         }
         __syncthreads();
         if (active)
             for (int kk = 0; kk < kc; ++kk)
                 decode_accumulate<B>(acc, a.packed + (int64_t)(k0 + kk) * p.packed_words + woff, table[kk]);
     }
-    if (!active) return;
+    if (!active) continue;
 
-    const float invK = __fdiv_rn(1.0f, (float)K);
     const int64_t base = L.elem_off + blk * kBlockCoords + 4 * lane;
     const int64_t limit = L.elem_off + L.size;
 #pragma unroll
@@ -103,22 +119,20 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
             if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
         }
     }
+    }
 }
 
 template <bool kQoda>
 __global__ void __launch_bounds__(kThreads) decode_kernel(PlanDev p, DecodeArgs a)
 {
-    __shared__ float table[kWorkerChunk][kMaxLevels];
+    __shared__ float table[kWorkerChunk][2 * kMaxLevels];
     const Tile tile = p.tiles[blockIdx.x];
     const int layer = tile.layer;
     const LayerDesc L = p.layers[layer];
-    const int warp = threadIdx.x >> 5;
-    const bool active = warp < tile.nblocks;
-    const int64_t blk = tile.block0 + warp;
     const float eta = kQoda ? p.scalars->eta : 0.0f;
 
     switch (L.bits) {
-#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kQoda>(p, L, layer, blk, active, a, table, eta); break;
+#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kQoda>(p, L, layer, tile, a, table, eta); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;

@@ -158,13 +158,16 @@ __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, cons
         if (s.moved <= 1e-13) break;
     }
 
-    // round to fp32; force strict monotonicity by single-ulp steps (serial: order matters)
+    // round to fp32; force strict monotonicity (one ulp and 2^-40 above the level before, one ulp
+    // below the level after; serial: order matters)
     if (tid == 0) {
         float* out = levels_stage + (int64_t)m * kLevelStride;
         out[0] = 0.0f; out[n - 1] = 1.0f;
         for (int j = 1; j <= n - 2; ++j) {
             const float f = (float)s.l[j];
-            const float fl = nextafterf(out[j - 1], 2.0f);
+            float fl = nextafterf(out[j - 1], 2.0f);
+            const float gap = __fadd_rn(out[j - 1], 9.094947017729282e-13f);   // previous level + 2^-40
+            if (gap > fl) fl = gap;
             out[j] = f > fl ? f : fl;
         }
         for (int j = n - 2; j >= 1; --j) {

@@ -9,10 +9,13 @@
 namespace lq {
 
 constexpr int kBlockCoords = 1024;    // coordinates per message block (32 lanes x 32 positions)
-constexpr int kTileBlocks = 8;        // blocks per tile = one per warp of a 256-thread CTA
+constexpr int kTileBlocks = 32;       // blocks per tile; the 8 warps of a CTA take them round-robin
+constexpr int kWarps = 8;
 constexpr int kThreads = 256;
 constexpr int kLevelStride = 256;     // floats per layer in a level table
 constexpr int kMaxLevels = 256;
+constexpr int kLutStride = 392;       // uint2 entries per layer in the search table (386 used)
+constexpr uint32_t kLutClamp = 0x33780000u;   // bit pattern one histogram bin below 2^-24
 
 struct LayerDesc {
     int64_t elem_off;     // first element of the layer inside a worker's fp32 row
@@ -60,14 +63,21 @@ struct PlanDev {
     QodaScalars* scalars;
 };
 
-struct lq_plan_impl;
-
 // ---- launchers (each enqueues on `s` and returns the launch status) ----
-cudaError_t launch_norm(const PlanDev& p, const float* grads, float* norms, cudaStream_t s);
+cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream_t s);
+cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
+// Encode-side tables derived from one level table (rebuilt whenever the levels change).
+struct SearchTables {
+    uint2* lut;        // [L][kLutStride]  {byte offset of tau0 in `ld`, bits of the level inside the bin or +inf}
+    float2* ld;        // [L][kMaxLevels]  {l_tau, (l_{tau+1} - l_tau) * 2^-24}
+    int32_t* fast;     // [L]              1 if every histogram bin holds at most one level
+};
+cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s);
 cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
                             const float* norms, uint32_t* hist, const uint32_t* prev_packed,
                             const float* prev_norms, const float* levels_cur,
-                            const float* levels_prev, cudaStream_t s);
+                            const float* levels_prev, SearchTables t, cudaStream_t s);
+cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
                           float* gbar, bool qoda, cudaStream_t s);

@@ -39,9 +39,10 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
 
     double acc = 0.0;
     uint32_t maxbits = 0;
-    if (warp < tile.nblocks) {
-        const int64_t base = (int64_t)(tile.block0 + warp) * kBlockCoords + 4 * lane;
-        if (base - 4 * lane + kBlockCoords <= L.size) {
+    for (int b = warp; b < tile.nblocks; b += kWarps) {
+        const int64_t blk0 = (int64_t)(tile.block0 + b) * kBlockCoords;
+        const int64_t base = blk0 + 4 * lane;
+        if (blk0 + kBlockCoords <= L.size) {
             float4 v[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -114,17 +115,19 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
     }
 }
 
-cudaError_t launch_norm(const PlanDev& p, const float* grads, float* norms, cudaStream_t s)
+cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream_t s)
 {
-    if (p.num_tiles > 0) {
-        const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
-        if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads);
-        else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads);
-        else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads);
-        else               norm_partial_kernel<3><<<grid, kThreads, 0, s>>>(p, grads);
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
+    if (p.num_tiles == 0) return cudaSuccess;
+    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
+    if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads);
+    else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads);
+    else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads);
+    else               norm_partial_kernel<3><<<grid, kThreads, 0, s>>>(p, grads);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s)
+{
     norm_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p, norms);
     return cudaGetLastError();
 }

@@ -234,30 +234,36 @@ def test_pack_roundtrip_all_widths_and_tails(orc):
 
 def test_pack_layout_hand_worked_positions(orc):
     """Positions worked out by hand from the layout text: block of 1024 coordinates, lane
-    (c/4)%32, position p = 4*(c/128) + c%4, plane 0 = signs, planes 1..b = code string."""
-    b = 3
+    (c/4)%32, position p = 4*(c/128) + c%4, symbol = sign*2^b + idx of b+1 bits at bit offset
+    p*(b+1) of the lane's string, bit t in word (t/32)*32 + lane."""
+    b = 3                                      # 4-bit symbols, 4 planes of 32 words per block
     d = 1200
     for (i, code, expect) in [
-        # i = 0: block 0, lane 0, p 0 -> sign bit 0 of word 0; code bits 0..2 of word 32
-        (0, 0b101, {0: 1 << 0, 32: 0b101}),
-        # i = 129: block 0, c = 129, lane (32)%32 = 0, p = 4*1 + 1 = 5 -> bits 15..17 of plane 1
-        (129, 0b111, {0: 1 << 5, 32: 0b111 << 15}),
-        # i = 7: lane 1, p = 3 -> bits 9..11 of plane 1, word 32 + 1
-        (7, 0b010, {1: 1 << 3, 33: 0b010 << 9}),
-        # i = 1023: lane 31, p = 4*7+3 = 31 -> bits 93..95 -> plane 3 (word 96+31) bits 29..31
-        (1023, 0b110, {31: 1 << 31, 96 + 31: 0b110 << 29}),
-        # i = 427: c = 427, lane (106)%32 = 10, p = 4*3 + 3 = 15 -> bit offset 45 -> plane 2 bits 13..15
-        (427, 0b011, {10: 1 << 15, 64 + 10: 0b011 << 13}),
-        # p = 10 (i = 2*128 + 4*lane + 2, lane 4 -> i = 274): offset 30 straddles planes 1 and 2
-        (274, 0b111, {4: 1 << 10, 32 + 4: 0b11 << 30, 64 + 4: 0b1}),
-        # second block: i = 1024 + 4 -> block base 128 words, lane 1, p 0
-        (1028, 0b001, {128 + 1: 1, 128 + 32 + 1: 0b001}),
+        # i = 0: block 0, lane 0, p 0 -> symbol 1101 in bits 0..3 of word 0
+        (0, 0b101, {0: 0b1101}),
+        # i = 129: c = 129, lane 32%32 = 0, p = 4*1+1 = 5 -> bits 20..23 of word 0
+        (129, 0b111, {0: 0b1111 << 20}),
+        # i = 7: lane 1, p = 3 -> bits 12..15 of word 1
+        (7, 0b010, {1: 0b1010 << 12}),
+        # i = 1023: lane 31, p = 31 -> bits 124..127 -> plane 3 (word 96+31) bits 28..31
+        (1023, 0b110, {96 + 31: 0b1110 << 28}),
+        # i = 427: lane 106%32 = 10, p = 4*3+3 = 15 -> bits 60..63 -> plane 1 (word 32+10) bits 28..31
+        (427, 0b011, {32 + 10: 0b1011 << 28}),
+        # second block: i = 1028 -> block base 128 words, lane 1, p 0
+        (1028, 0b001, {128 + 1: 0b1001}),
     ]:
         idx = np.zeros(d, np.uint8); sg = np.zeros(d, np.uint8)
         idx[i] = code; sg[i] = 1
         w = orc.pack_layer(idx, sg, b)
         got = {int(j): int(w[j]) for j in np.flatnonzero(w)}
         assert got == expect, (i, got, expect)
+    # b = 4: 5-bit symbols straddle words; p = 6 (i = 128 + 4*lane + 2, lane 3 -> i = 142) sits at
+    # bits 30..34: two bits in plane 0 and three in plane 1
+    idx = np.zeros(200, np.uint8); sg = np.zeros(200, np.uint8)
+    idx[142] = 0b1011; sg[142] = 1                  # symbol 11011
+    w = orc.pack_layer(idx, sg, 4)
+    got = {int(j): int(w[j]) for j in np.flatnonzero(w)}
+    assert got == {3: 0b11 << 30, 32 + 3: 0b110}
 
 
 # ---------------------------------------------------------------------------- histogram
