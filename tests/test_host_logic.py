@@ -1,0 +1,103 @@
+"""CPU-only checks of the host side: the C-ABI library loads and exports every symbol the header
+declares, and the benchmark's multi-rank bookkeeping (max over ranks, whole-job value) works
+across two gloo ranks.  No kernel is launched here.
+"""
+import ctypes
+import json
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "lq.h")
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)             # drop comments
+    text = re.sub(r"^\s*#.*$", "", text, flags=re.M)              # drop preprocessor lines
+    names = re.findall(r"\b([a-z_][a-z0-9_]*)\s*\([^;{]*\)\s*;", text)
+    return sorted(set(names))
+
+
+def test_header_declares_the_named_entry_points():
+    names = _declared_functions()
+    for required in ["lq_plan_create", "lq_fit_levels", "lq_quantize_pack", "lq_decode_aggregate", "qoda_step"]:
+        assert required in names
+    assert len(names) >= 19
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    from paper_2505_14371_b200 import build as b
+    path = b.build()
+    lib = ctypes.CDLL(path)
+    for name in _declared_functions():
+        assert hasattr(lib, name), f"liblq.so does not export {name}"
+    # the binding declares the same set
+    from paper_2505_14371_b200 import binding
+    assert sorted(binding.EXPORTS) == _declared_functions()
+    # entry points that touch no device
+    lib.lq_error_string.restype = ctypes.c_char_p
+    assert lib.lq_error_string(0) == b"ok"
+    assert lib.lq_error_string(-1) == b"invalid argument"
+    lib.lq_plan_padded_elems.restype = ctypes.c_int64
+    lib.lq_plan_padded_elems.argtypes = [ctypes.c_void_p]
+    assert lib.lq_plan_padded_elems(None) == -1                   # LQ_EINVAL, reported not crashed
+    assert lib.lq_plan_destroy(None) == 0
+
+
+def test_binding_has_no_cpu_fallback(monkeypatch):
+    from paper_2505_14371_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", os.path.join(ROOT, "does_not_exist", "liblq.so"))
+    with pytest.raises(binding.LqError):
+        binding.load_library()
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2505_14371_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src.lower().replace("cpu oracle", ""), f
+
+
+_RANK_SCRIPT = r"""
+import json, os, sys
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+local_ms = 2.0 if rank == 0 else 5.0            # rank 1 is the slow one
+ms = bench.aggregate_over_ranks(local_ms, world)
+value = bench.whole_job_value(10.0, world, ms)
+open(os.path.join({out!r}, "rank%d.json" % rank), "w").write(json.dumps({{"rank": rank, "ms": ms, "value": value}}))
+dist.destroy_process_group()
+"""
+
+
+def test_two_gloo_ranks_take_the_max_time_and_sum_the_units(tmp_path):
+    script = tmp_path / "rank.py"
+    script.write_text(_RANK_SCRIPT.format(root=ROOT, out=str(tmp_path)))
+    port = 29500 + os.getpid() % 2000
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+                          "--master-addr", "127.0.0.1", "--master-port", str(port), str(script)],
+                         capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    rows = [json.loads((tmp_path / f"rank{r}.json").read_text()) for r in range(2)]
+    assert sorted(r["rank"] for r in rows) == [0, 1]
+    for r in rows:
+        assert r["ms"] == 5.0                                     # max over ranks
+        assert abs(r["value"] - 2 * 10.0 / 5e-3) < 1e-9           # all ranks' units / slowest rank's time
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2")
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
+                         capture_output=True, text=True, timeout=120, env=env)
+    assert out.returncode == 0 and out.stdout.strip() == ""
