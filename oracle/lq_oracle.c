@@ -51,14 +51,15 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
 
 /* Uniform in [0,1) for coordinate `index` of (worker, layer) at iteration `step`:
  * key = (seed low, seed high), counter = (index / 4, layer, worker, step), the coordinate
- * takes output word index % 4, and rho = (word >> 8) * 2^-24 (exact in fp32). */
+ * takes output word index % 4, and rho = (word >> 9) * 2^-23: the top 23 bits of the word
+ * on the grid of fp32 numbers in [0,1) with spacing 2^-23 (exact in fp32). */
 float orc_uniform(uint64_t seed, uint32_t step, uint32_t worker, uint32_t layer, uint64_t index)
 {
     uint32_t ctr[4] = { (uint32_t)(index >> 2), layer, worker, step };
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
-    return (float)(out[index & 3] >> 8) * 5.9604644775390625e-08f; /* 2^-24 */
+    return (float)(out[index & 3] >> 9) * 1.1920928955078125e-07f; /* 2^-23 */
 }
 
 /* ------------------------------------------------------------------------------------
@@ -98,7 +99,7 @@ float orc_layer_norm(const float* v, int64_t d, int q, int* status)
  *   tau = the largest j <= n-2 with level[j] <= u   (so u = 1 falls in the last interval)
  *   up with probability xi(u) = (u - l_tau) / (l_{tau+1} - l_tau), decided as
  *        rho * (l_{tau+1} - l_tau) < (u - l_tau)     with rho the coordinate's uniform
- *   idx = tau + up,  sign = sign bit of v.
+ *   idx = tau + up,  sign = (v < 0), so both zeros carry sign 0.
  * `near` counts coordinates whose decision is within 1e-6 (relative to the interval)
  * of the threshold.  norm == 0 gives an all-zero message.
  * v points at coordinate `first_index` of the layer and d coordinates are processed, so
@@ -129,7 +130,7 @@ void orc_quantize_layer(const float* v, int64_t d, int64_t first_index, float no
         int up = (t < num) ? 1 : 0;
         if (fabsf(t - num) <= 1e-6f * den) ++near_count;
         idx[i] = (uint8_t)(tau + up);
-        sign[i] = (uint8_t)(signbit(v[i]) ? 1 : 0);
+        sign[i] = (uint8_t)(v[i] < 0.0f ? 1 : 0);
     }
     if (near) *near = near_count;
 }
@@ -417,14 +418,16 @@ void orc_aggregate(const float* decoded, int K, int64_t d, float* gbar)
     }
 }
 
-/* sum_i (cur_i - prev_i)^2 in fp64 with exact differences: one worker-layer term of the
- * adaptive step size (Eq. general_stepsize: ||V^_{k,s+1/2} - V^_{k,s-1/2}||^2). */
+/* One worker-layer term of the adaptive step size (Eq. general_stepsize:
+ * ||V^_{k,s+1/2} - V^_{k,s-1/2}||^2).  The decoded vectors are fp32, and their difference is
+ * formed in that precision (one fp32 subtraction per coordinate); the squares of those fp32
+ * differences, exact in fp64, are summed in fp64. */
 double orc_sq_diff(const float* cur, const float* prev, int64_t d)
 {
     double acc = 0.0;
     for (int64_t i = 0; i < d; ++i) {
-        double t = (double)cur[i] - (prev ? (double)prev[i] : 0.0);
-        acc += t * t;
+        float t = cur[i] - (prev ? prev[i] : 0.0f);
+        acc += (double)t * (double)t;
     }
     return acc;
 }

@@ -12,18 +12,6 @@ namespace lq {
 
 constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
 
-// symbol p (pre-scaled by 4) of a lane's string of 32 symbols of C bits, held in C words
-template <int C>
-__device__ __forceinline__ uint32_t symbol4_at(const uint32_t (&w)[C], int p)
-{
-    const int off = p * C, i = off >> 5, s = off & 31;
-    constexpr uint32_t mask4 = ((1u << C) - 1u) << 2;
-    uint32_t v;
-    if (s + C <= 32) v = s >= 2 ? (w[i] >> (s - 2)) : (w[i] << (2 - s));
-    else             v = __funnelshift_r(w[i], w[i + 1], s - 2);      // s >= 2 whenever a symbol straddles
-    return v & mask4;
-}
-
 // Adds one worker's decoded block into acc.  `table` holds N * l_j for j < n and -N * l_j after.
 template <int B>
 __device__ __forceinline__ void decode_accumulate(float (&acc)[32], const uint32_t* __restrict__ words,

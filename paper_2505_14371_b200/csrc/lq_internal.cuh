@@ -68,8 +68,8 @@ cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
 // Encode-side tables derived from one level table (rebuilt whenever the levels change).
 struct SearchTables {
-    uint2* lut;        // [L][kLutStride]  {byte offset of tau0 in `ld`, bits of the level inside the bin or +inf}
-    float2* ld;        // [L][kMaxLevels]  {l_tau, (l_{tau+1} - l_tau) * 2^-24}
+    uint2* lut;        // [L][kLutStride]  {4 * tau0, bits of the level inside the bin or +inf}
+    float2* ld;        // [L][kMaxLevels]  {l_tau, l_{tau+1} - l_tau}
     int32_t* fast;     // [L]              1 if every histogram bin holds at most one level
 };
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s);
@@ -109,6 +109,18 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
         k1 += 0xBB67AE85u;
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// symbol p (pre-scaled by 4) of a lane's string of 32 symbols of C bits, held in C words
+template <int C>
+__device__ __forceinline__ uint32_t symbol4_at(const uint32_t (&w)[C], int p)
+{
+    const int off = p * C, i = off >> 5, s = off & 31;
+    constexpr uint32_t mask4 = ((1u << C) - 1u) << 2;
+    uint32_t v;
+    if (s + C <= 32) v = s >= 2 ? (w[i] >> (s - 2)) : (w[i] << (2 - s));
+    else             v = __funnelshift_r(w[i], w[i + 1], s - 2);      // s >= 2 whenever a symbol straddles
+    return v & mask4;
 }
 
 __device__ __forceinline__ double warp_sum(double v)

@@ -5,157 +5,229 @@
 //
 // Work decomposition: one CTA per (tile, worker); a tile is up to 32 blocks of 1024 coordinates of
 // one layer, taken round-robin by the 8 warps.  A lane owns the 32 coordinates {128 j + 4 lane + e}
-// of a block: it reads them as 8 coalesced float4 loads, draws one Philox4x32-10 block per float4
-// (4 uniforms) and ends up with exactly b+1 words of symbols, which it stores plane by plane so
-// that a warp writes 128 contiguous bytes per plane.  No shuffles, ballots or atomics on the
-// main path.
+// of a block (row j = one float4 per lane, 512 contiguous bytes per warp).  Rows travel from global
+// memory into a per-warp ring of 8 rows in shared memory with 16-byte asynchronous copies, so a
+// warp always has 4 KB in flight and the values never sit in registers while they wait; every lane
+// reads back only the bytes it copied itself, so the ring needs no barrier.  Per row the lane draws
+// one Philox4x32-10 block (4 uniforms); after 8 rows it holds exactly b+1 words of symbols, which it
+// stores plane by plane (128 contiguous bytes per warp and plane).  No shuffles, ballots or atomics
+// on the main path.
 //
-// The level search uses a table over the 386 histogram bins of u (exponent + 4 mantissa bits):
-// each entry names the last level at or below the bin's lower edge and the single level that may
-// lie inside the bin, so tau costs one shared-memory load and one compare.  Layers whose levels
-// are denser than the bins fall back to a binary search.  All byte offsets are kept pre-scaled by
-// 8 so that the same register indexes the {level, gap} table and the fp64 value tables.
+// The level search uses a table over the 386 histogram bins of u (exponent + 4 mantissa bits): each
+// entry names the last level at or below the bin's lower edge and the single level that may lie
+// inside the bin, so tau costs one shared-memory load and one compare.  Layers whose levels are
+// denser than the bins fall back to a binary search.  Levels, gaps and the decoded values of the
+// current and the previous message sit in 4-byte tables (conflict-free up to 32 entries); all table
+// offsets are kept pre-scaled by 4.
+//
+// A row whose 128 values are all +0 (untouched embedding rows, zeroed layers) skips the random
+// numbers and the search: its symbols are 0.  If the previous message is all zero there as well,
+// the row adds nothing to the statistic and is skipped entirely.
 #include "lq_internal.cuh"
 
 namespace lq {
 
+constexpr int kRingRows = 8;                       // rows of 512 bytes in flight per warp
+constexpr int kRingBytes = kWarps * kRingRows * 512;
+
 struct QuantSmem {
-    uint2 lut[kLutStride];           // search table of this layer
-    float2 ld[kMaxLevels];           // {l_tau, (l_{tau+1}-l_tau) * 2^-24}
-    float lev[kMaxLevels];           // plain levels (binary-search path)
-    double tcur[2 * kMaxLevels];     // (double) fp32(N_cur * l_j), second half negated
-    double tprev[2 * kMaxLevels];    // same for the previous message
+    uint2 lut[kLutStride];           // search table of this layer: {4 * tau0, boundary bits}
+    float lev[kMaxLevels];           // l_tau
+    float gap[kMaxLevels];           // l_{tau+1} - l_tau
+    float tcur[2 * kMaxLevels];      // fp32(N_cur * l_j) by symbol, second half negated
+    float tprev[2 * kMaxLevels];     // same for the previous message
     uint32_t hist[LQ_HIST_STRIDE];
     double scratch[kWarps];
 };
 
-// symbol p (pre-scaled by 8) of a lane's string of 32 symbols of C bits, held in C words
-template <int C>
-__device__ __forceinline__ uint32_t symbol8_at(const uint32_t (&w)[C], int p)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes)
 {
-    const int off = p * C, i = off >> 5, s = off & 31;
-    constexpr uint32_t mask8 = ((1u << C) - 1u) << 3;
-    uint32_t v;
-    if (s + C <= 32) v = s >= 3 ? (w[i] >> (s - 3)) : (w[i] << (3 - s));
-    else             v = __funnelshift_r(w[i], w[i + 1], s - 3);      // s >= 3 whenever a symbol straddles
-    return v & mask8;
+    // copies `bytes` (0..16) bytes and fills the rest of the 16 with zeros
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int C>
-__device__ __forceinline__ void put_symbol8(uint32_t (&w)[C], int p, uint32_t sym8)
+__device__ __forceinline__ void put_symbol4(uint32_t (&w)[C], int p, uint32_t sym4)
 {
     const int off = p * C, i = off >> 5, s = off & 31;
-    w[i] += s >= 3 ? (sym8 << (s - 3)) : (sym8 >> (3 - s));           // fields never overlap: + is |
-    if (s + C > 32) w[i + 1] = sym8 >> (35 - s);
+    w[i] += s >= 2 ? (sym4 << (s - 2)) : (sym4 >> (2 - s));           // fields never overlap: + is |
+    if (s + C > 32) w[i + 1] = sym4 >> (34 - s);
+}
+
+// Everything a warp needs to walk its blocks of one (tile, worker).
+struct WarpCtx {
+    const float* g;              // first coordinate of the layer in this worker's row
+    int64_t size;                // d_m
+    uint32_t ring;               // shared-memory address of this lane's 16 bytes in ring row 0
+    const float4* ring_ptr;      // the same place as a pointer
+    float r;                     // 1/N, or 0 for a zeroed layer
+    int lane;
+};
+
+// Starts the copy of row j of block `blk` into ring row j (zero-filled past the layer's end).
+__device__ __forceinline__ void issue_row(const WarpCtx& c, int64_t blk, int j)
+{
+    const int64_t pos = blk * kBlockCoords + 128 * j + 4 * c.lane;
+    const int64_t rem = c.size - pos;
+    const int bytes = rem >= 4 ? 16 : (rem > 0 ? 4 * (int)rem : 0);
+    cp_async16(c.ring + 512u * j, rem > 0 ? c.g + pos : c.g, bytes);
 }
 
 template <int B, bool kFast, bool kHist>
-__device__ __forceinline__ double quantize_block(const PlanDev& p, const LayerDesc& L, int layer, int k,
-                                                 int64_t blk, const float* __restrict__ g, float r,
-                                                 uint32_t step, uint32_t* __restrict__ out,
-                                                 const uint32_t* __restrict__ prev, QuantSmem& sm)
+__device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx& c, int layer, int k,
+                                                 int64_t blk, bool has_next, uint32_t step,
+                                                 uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
+                                                 bool prev_live, QuantSmem& sm)
 {
     constexpr int n = 1 << B, C = B + 1;
-    const int lane = threadIdx.x & 31;
-    const int64_t base = blk * kBlockCoords + 4 * lane;
-
-    float4 v[8];
-    if (r == 0.0f) {
+    const int lane = c.lane;
+    const float r = c.r;
+    uint32_t cw[C];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    } else if (blk * kBlockCoords + kBlockCoords <= L.size) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = __ldcs(reinterpret_cast<const float4*>(g + base + 128 * j));
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int64_t pos = base + 128 * j;
-            v[j].x = pos + 0 < L.size ? __ldg(g + pos + 0) : 0.f;
-            v[j].y = pos + 1 < L.size ? __ldg(g + pos + 1) : 0.f;
-            v[j].z = pos + 2 < L.size ? __ldg(g + pos + 2) : 0.f;
-            v[j].w = pos + 3 < L.size ? __ldg(g + pos + 3) : 0.f;
-        }
-    }
-
-    const int64_t woff = blk * (int64_t)C * 32 + lane;
-    uint32_t pw[C], cw[C];
-#pragma unroll
-    for (int w = 0; w < C; ++w) { pw[w] = prev ? __ldcs(prev + woff + w * 32) : 0u; cw[w] = 0u; }
+    for (int w = 0; w < C; ++w) cw[w] = 0u;
 
     const char* lut_b = reinterpret_cast<const char*>(sm.lut) - (kLutClamp >> 16);
-    const char* ld_b = reinterpret_cast<const char*>(sm.ld);
+    const char* lev_b = reinterpret_cast<const char*>(sm.lev);
+    const char* gap_b = reinterpret_cast<const char*>(sm.gap);
     const char* tcur_b = reinterpret_cast<const char*>(sm.tcur);
     const char* tprev_b = reinterpret_cast<const char*>(sm.tprev);
     double stat = 0.0;
 
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        uint32_t x[4];
-        philox4x32_10((uint32_t)(blk * 256 + 32 * j + lane), (uint32_t)layer, (uint32_t)k, step,
-                      p.seed_lo, p.seed_hi, x);
-        const float vv[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+    for (int j = 0; j < kRingRows; ++j) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r != 0.0f) {
+            cp_async_wait<kRingRows - 1>();
+            v = c.ring_ptr[32 * j];
+            // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
+            v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
+            v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
+        }
+        const float vv[4] = {v.x, v.y, v.z, v.w};
+        const uint32_t any_bits = __float_as_uint(v.x) | __float_as_uint(v.y) | __float_as_uint(v.z) |
+                                  __float_as_uint(v.w);
+        if (kHist || __any_sync(0xffffffffu, any_bits != 0u)) {
+            uint32_t x[4];
+            philox4x32_10((uint32_t)(blk * 256 + 32 * j + lane), (uint32_t)layer, (uint32_t)k, step,
+                          p.seed_lo, p.seed_hi, x);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int pp = 4 * j + e;
-            const uint32_t bits = __float_as_uint(vv[e]);
-            // u <= 1 + 2^-23 always (N >= |v| and one rounding each in 1/N and the product), and
-            // such a u behaves exactly like u = 1 below, so the min(u, 1) of the definition is not needed
-            const float u = __fmul_rn(fabsf(vv[e]), r);
-            const uint32_t ub = __float_as_uint(u);
-            uint32_t t8;
-            if (kFast) {
-                const uint32_t off = (max(ub, kLutClamp) >> 16) & ~7u;
-                const uint2 en = *reinterpret_cast<const uint2*>(lut_b + off);
-                t8 = en.x + (u >= __uint_as_float(en.y) ? 8u : 0u);
-            } else {
-                int tau = 0;
+            for (int e = 0; e < 4; ++e) {
+                const int pp = 4 * j + e;
+                const uint32_t bits = __float_as_uint(vv[e]);
+                // u <= 1 + 2^-23 always (N >= |v| and one rounding each in 1/N and the product), and
+                // such a u behaves exactly like u = 1 below, so the min(u, 1) of the definition is not needed
+                const float u = __fmul_rn(fabsf(vv[e]), r);
+                const uint32_t ub = __float_as_uint(u);
+                uint32_t t4;
+                if (kFast) {
+                    const uint32_t off = (max(ub, kLutClamp) >> 16) & ~7u;
+                    const uint2 en = *reinterpret_cast<const uint2*>(lut_b + off);
+                    t4 = en.x + (u >= __uint_as_float(en.y) ? 4u : 0u);
+                } else {
+                    int tau = 0;
 #pragma unroll
-                for (int s = B - 1; s >= 0; --s) {
-                    const int cand = tau + (1 << s);
-                    if (sm.lev[cand] <= u) tau = cand;
+                    for (int s = B - 1; s >= 0; --s) {
+                        const int cand = tau + (1 << s);
+                        if (sm.lev[cand] <= u) tau = cand;
+                    }
+                    t4 = 4u * (uint32_t)min(tau, n - 2);
                 }
-                t8 = 8u * (uint32_t)min(tau, n - 2);
-            }
-            const float2 ld = *reinterpret_cast<const float2*>(ld_b + t8);
-            const float num = __fsub_rn(u, ld.x);
-            const float rho = __uint2float_rn(x[e] >> 8);                 // 2^24 * uniform, exact
-            const uint32_t i8 = t8 + (__fmul_rn(rho, ld.y) < num ? 8u : 0u);
-            const uint32_t sym8 = i8 + (bits >> 31) * (8u * n);
-            put_symbol8<C>(cw, pp, sym8);
+                const float l0 = *reinterpret_cast<const float*>(lev_b + t4);
+                const float den = *reinterpret_cast<const float*>(gap_b + t4);
+                const float num = __fsub_rn(u, l0);
+                // rho = (x >> 9) * 2^-23; f = 1 + rho is built from the bits, and fma(f, den, -den)
+                // rounds the exact product rho * den once, like the plain multiplication
+                const float f = __uint_as_float(__funnelshift_r(x[e], 0x7Fu, 9));
+                const float t = __fmaf_rn(f, den, -den);
+                const uint32_t i4 = t4 + (t < num ? 4u : 0u);
+                const uint32_t sym4 = i4 | ((bits >> (29 - B)) & (4u * n));
+                put_symbol4<C>(cw, pp, sym4);
 
-            if (kHist) {
-                const int64_t pos = base + 128 * j + e;
-                if (r != 0.0f && pos < L.size)
-                    atomicAdd(&sm.hist[(max(ub, kLutClamp) - kLutClamp) >> 19], 1u);
-            }
+                if (kHist) {
+                    const int64_t pos = blk * kBlockCoords + 128 * j + 4 * lane + e;
+                    if (r != 0.0f && pos < c.size)
+                        atomicAdd(&sm.hist[(max(ub, kLutClamp) - kLutClamp) >> 19], 1u);
+                }
 
-            // step-size statistic: exact fp64 difference of the two fp32 decoded values
-            const double cur = *reinterpret_cast<const double*>(tcur_b + sym8);
-            const double prv = *reinterpret_cast<const double*>(tprev_b + symbol8_at<C>(pw, pp));
-            const double dd = cur - prv;
-            stat = fma(dd, dd, stat);
+                // step-size statistic: fp32 difference of the two decoded values, squared in fp64
+                const float cur = *reinterpret_cast<const float*>(tcur_b + sym4);
+                const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, pp));
+                const double dd = (double)__fsub_rn(cur, prv);
+                stat = fma(dd, dd, stat);
+            }
+        } else if (prev_live) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, 4 * j + e));
+                const double dd = (double)__fsub_rn(0.0f, prv);
+                stat = fma(dd, dd, stat);
+            }
+        }
+        if (r != 0.0f) {
+            if (has_next) issue_row(c, blk + kWarps, j);
+            cp_async_commit();
         }
     }
+    const int64_t woff = blk * (int64_t)C * 32 + lane;
 #pragma unroll
     for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, cw[w]);
     return stat;
 }
 
+template <int B, bool kFast, bool kHist>
+__device__ __forceinline__ double quantize_tile(const PlanDev& p, const WarpCtx& c, const Tile& tile, int layer,
+                                                int k, uint32_t step, uint32_t* __restrict__ out,
+                                                const uint32_t* __restrict__ prev, QuantSmem& sm)
+{
+    constexpr int C = B + 1;
+    const int warp = threadIdx.x >> 5;
+    double stat = 0.0;
+    if (warp >= tile.nblocks) return stat;
+    int64_t blk = tile.block0 + warp;
+    const int64_t end = tile.block0 + tile.nblocks;
+    if (c.r != 0.0f) {
+#pragma unroll
+        for (int j = 0; j < kRingRows; ++j) { issue_row(c, blk, j); cp_async_commit(); }
+    }
+    uint32_t pw[C];
+#pragma unroll
+    for (int w = 0; w < C; ++w) pw[w] = prev ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
+    for (; blk < end; blk += kWarps) {
+        const bool has_next = blk + kWarps < end;
+        uint32_t pn[C];                                   // the next block's previous words, fetched early
+#pragma unroll
+        for (int w = 0; w < C; ++w)
+            pn[w] = (prev && has_next) ? __ldcs(prev + (blk + kWarps) * (int64_t)C * 32 + c.lane + w * 32) : 0u;
+        uint32_t por = 0u;
+#pragma unroll
+        for (int w = 0; w < C; ++w) por |= pw[w];
+        const bool prev_live = __any_sync(0xffffffffu, por != 0u);
+        stat += quantize_block<B, kFast, kHist>(p, c, layer, k, blk, has_next, step, out, pw, prev_live, sm);
+#pragma unroll
+        for (int w = 0; w < C; ++w) pw[w] = pn[w];
+    }
+    cp_async_wait<0>();
+    return stat;
+}
+
 template <bool kHist>
-__global__ void __launch_bounds__(kThreads) quantize_pack_kernel(
+__global__ void __launch_bounds__(kThreads, 3) quantize_pack_kernel(
     PlanDev p, const float* __restrict__ grads, uint32_t step, uint32_t* __restrict__ packed,
     const float* __restrict__ norms, uint32_t* __restrict__ hist,
     const uint32_t* __restrict__ prev_packed, const float* __restrict__ prev_norms,
     const float* __restrict__ levels_cur, const float* __restrict__ levels_prev, SearchTables st)
 {
     __shared__ QuantSmem sm;
+    extern __shared__ float4 ring_mem[];              // [warp][row][lane] float4
     const Tile tile = p.tiles[blockIdx.x];
     const int layer = tile.layer;
     const LayerDesc L = p.layers[layer];
     const int k = blockIdx.y;
-    const int warp = threadIdx.x >> 5;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t kl = (int64_t)k * p.num_layers + layer;
-    const float r = p.rnorm[kl];
     const float ncur = norms[kl];
     const float nprev = prev_norms ? prev_norms[kl] : 0.0f;
     const bool fast = st.fast[layer] != 0;
@@ -163,10 +235,11 @@ __global__ void __launch_bounds__(kThreads) quantize_pack_kernel(
 
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const float l = levels_cur[(int64_t)layer * kLevelStride + i];
-        const double c = (double)__fmul_rn(ncur, l);
-        const double q = (double)__fmul_rn(nprev, levels_prev[(int64_t)layer * kLevelStride + i]);
-        sm.lev[i] = l;
-        sm.ld[i] = st.ld[(int64_t)layer * kMaxLevels + i];
+        const float c = __fmul_rn(ncur, l);
+        const float q = __fmul_rn(nprev, levels_prev[(int64_t)layer * kLevelStride + i]);
+        const float2 ld = st.ld[(int64_t)layer * kMaxLevels + i];
+        sm.lev[i] = fast ? ld.x : l;                  // the binary search reads plain levels, all n of them
+        sm.gap[i] = ld.y;
         sm.tcur[i] = c;  sm.tcur[n + i] = -c;
         sm.tprev[i] = q; sm.tprev[n + i] = -q;
     }
@@ -177,21 +250,24 @@ __global__ void __launch_bounds__(kThreads) quantize_pack_kernel(
         for (int i = threadIdx.x; i < LQ_HIST_STRIDE; i += blockDim.x) sm.hist[i] = 0;
     __syncthreads();
 
-    const float* g = grads + (int64_t)k * p.padded_elems + L.elem_off;
+    WarpCtx c;
+    c.g = grads + (int64_t)k * p.padded_elems + L.elem_off;
+    c.size = L.size;
+    c.ring_ptr = ring_mem + (warp * kRingRows) * 32 + lane;
+    c.ring = (uint32_t)__cvta_generic_to_shared(c.ring_ptr);
+    c.r = p.rnorm[kl];
+    c.lane = lane;
     uint32_t* out = packed + (int64_t)k * p.packed_words + L.word_off;
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
 
     double stat = 0.0;
-    for (int b = warp; b < tile.nblocks; b += kWarps) {
-        const int64_t blk = tile.block0 + b;
-        switch (L.bits * 2 + (fast ? 1 : 0)) {
-#define LQ_CASE(BB)                                                                                       \
-    case 2 * BB:     stat += quantize_block<BB, false, kHist>(p, L, layer, k, blk, g, r, step, out, prev, sm); break; \
-    case 2 * BB + 1: stat += quantize_block<BB, true, kHist>(p, L, layer, k, blk, g, r, step, out, prev, sm); break;
-            LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
+    switch (L.bits * 2 + (fast ? 1 : 0)) {
+#define LQ_CASE(BB)                                                                                   \
+    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(p, c, tile, layer, k, step, out, prev, sm); break; \
+    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(p, c, tile, layer, k, step, out, prev, sm); break;
+        LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
-            default: break;
-        }
+        default: break;
     }
     const double total = block_reduce<false>(stat, sm.scratch);
     if (threadIdx.x == 0) p.stat_partial[(int64_t)k * p.num_tiles + blockIdx.x] = total;
@@ -218,8 +294,8 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 }
 
 // One CTA per layer: derives the encode-side tables from the layer's levels.
-//   ld[tau]  = {l_tau, (l_{tau+1} - l_tau) * 2^-24}       tau = 0..n-2
-//   lut[bin] = {8 * tau0, bits of l_{tau0+1} if it lies inside the bin, else +inf}
+//   ld[tau]  = {l_tau, l_{tau+1} - l_tau}                 tau = 0..n-2 (other entries: {l_tau, 0})
+//   lut[bin] = {4 * tau0, bits of l_{tau0+1} if it lies inside the bin, else +inf}
 //              tau0 = last level (<= n-2) at or below the bin's lower edge
 //   fast     = no bin holds two or more levels (then tau is tau0 or tau0 + 1)
 __global__ void __launch_bounds__(128) build_search_kernel(PlanDev p, const float* __restrict__ levels,
@@ -233,8 +309,8 @@ __global__ void __launch_bounds__(128) build_search_kernel(PlanDev p, const floa
     for (int i = threadIdx.x; i < n; i += blockDim.x) lev[i] = levels[(int64_t)m * kLevelStride + i];
     __syncthreads();
     for (int i = threadIdx.x; i < kMaxLevels; i += blockDim.x) {
-        float2 e = make_float2(0.f, 0.f);
-        if (i <= n - 2) e = make_float2(lev[i], __fmul_rn(__fsub_rn(lev[i + 1], lev[i]), 5.9604644775390625e-08f));
+        float2 e = make_float2(i < n ? lev[i] : 0.f, 0.f);
+        if (i <= n - 2) e.y = __fsub_rn(lev[i + 1], lev[i]);
         t.ld[(int64_t)m * kMaxLevels + i] = e;
     }
     for (int bin = threadIdx.x; bin < LQ_NUM_BINS; bin += blockDim.x) {
@@ -247,7 +323,7 @@ __global__ void __launch_bounds__(128) build_search_kernel(PlanDev p, const floa
             boundary = __float_as_uint(lev[tau0 + 1]);
             if (tau0 + 2 <= n - 2 && lev[tau0 + 2] < hi) atomicOr(&slow, 1);
         }
-        t.lut[(int64_t)m * kLutStride + bin] = make_uint2(8u * (uint32_t)tau0, boundary);
+        t.lut[(int64_t)m * kLutStride + bin] = make_uint2(4u * (uint32_t)tau0, boundary);
     }
     __syncthreads();
     if (threadIdx.x == 0) t.fast[m] = slow ? 0 : 1;
@@ -268,10 +344,10 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
     if (p.num_tiles == 0) return cudaSuccess;
     const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
     if (hist)
-        quantize_pack_kernel<true><<<grid, kThreads, 0, s>>>(p, grads, step, packed, norms, hist, prev_packed,
+        quantize_pack_kernel<true><<<grid, kThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist, prev_packed,
                                                              prev_norms, levels_cur, levels_prev, t);
     else
-        quantize_pack_kernel<false><<<grid, kThreads, 0, s>>>(p, grads, step, packed, norms, hist, prev_packed,
+        quantize_pack_kernel<false><<<grid, kThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist, prev_packed,
                                                               prev_norms, levels_cur, levels_prev, t);
     return cudaGetLastError();
 }

@@ -143,6 +143,32 @@ def test_statistic_with_previous_message_and_level_change(lqm, orc):
         assert _close(sq.numpy(), ref["sq_diff"], 1e-12), step
 
 
+def test_zero_rows_and_negative_zero(lqm, orc):
+    """Long runs of +0 and -0 (rows nobody touched): symbols 0, sign 0, and the statistic still sees
+    the previous message where the current one is zero."""
+    sizes = [9000, 70001, 300]
+    plan = lqm.Plan(sizes, [4, 3, 4], 2, 2, SEED)
+    model = oracle_model(orc, plan)
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    o = plan.elem_offsets
+    for step in range(1, 4):
+        grads = _grads(plan, 40 + step, 0.3)
+        a = 1024 * step
+        grads[:, o[0] + a: o[0] + a + 3000] = 0.0
+        grads[0, o[1] + 100: o[1] + 60000] *= 0.0          # leaves -0.0 where the value was negative
+        grads[1, o[1] + 30000 + 128 * step: o[1] + 30000 + 128 * step + 4096] = -0.0
+        if step == 3:
+            grads[:, o[2]: o[2] + 300] = -0.0               # a whole layer of -0: zero norm
+        c, p = step % 2, (step + 1) % 2
+        plan.lq_quantize_pack(grads, step, pk[c], nm[c], prev_packed=None if step == 1 else pk[p],
+                              prev_norms=None if step == 1 else nm[p])
+        ref = model.quantize(to_unpadded(plan, grads), step)
+        model.prev_decoded = ref["decoded"]
+        assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+        sq, _ = plan.lq_get_statistics()
+        assert _close(sq.numpy(), ref["sq_diff"], 1e-12), step
+
+
 @pytest.mark.parametrize("K", [1, 4, 11, 16])
 def test_decode_aggregate_worker_counts(lqm, orc, K):
     sizes = [4100, 7, 1024, 2049]

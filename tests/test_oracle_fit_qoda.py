@@ -169,6 +169,10 @@ def test_step_size_formula(orc):
     assert S == 3.0 and eta == np.float32(0.5)
     a = np.float32([1.0, 2.0, -3.0]); b = np.float32([0.5, 2.0, 1.0])
     assert orc.sq_diff(a, b) == 0.25 + 16.0 and orc.sq_diff(a, None) == 14.0
+    # the difference is an fp32 subtraction (the vectors' own precision), its square summed in fp64
+    assert orc.sq_diff(np.float32([1.0]), np.float32([2.0 ** -30])) == 1.0
+    big = np.float32([3.0] * 4 + [2.0 ** -20]); zero = np.zeros(5, np.float32)
+    assert orc.sq_diff(big, zero) == 36.0 + 2.0 ** -40          # fp64 accumulation keeps the small term
 
 
 def test_qoda_identities_with_quantization(orc):

@@ -33,7 +33,7 @@ def test_uniform_keying_and_range(orc):
     for (step, worker, layer, i) in [(0, 0, 0, 0), (7, 3, 2, 5), (2 ** 32 - 1, 15, 224, 2 ** 33 + 3)]:
         out = orc.philox4x32_10([(i >> 2) & 0xFFFFFFFF, layer, worker, step],
                                 [seed & 0xFFFFFFFF, seed >> 32])
-        assert orc.uniform(seed, step, worker, layer, i) == (out[i & 3] >> 8) / 2.0 ** 24
+        assert orc.uniform(seed, step, worker, layer, i) == (out[i & 3] >> 9) / 2.0 ** 23
     u = np.array([orc.uniform(SEED, 1, 0, 0, i) for i in range(20000)])
     assert u.min() >= 0.0 and u.max() < 1.0
     # mean and variance of U(0,1), lag-1 correlation
@@ -202,6 +202,13 @@ def test_uniform_levels_reduce_to_floor_plus_bernoulli(orc):
     for s in range(R):
         acc += orc.quantize_layer(v, norm, levels, SEED, 1000 + s, 0, 0)[0]
     assert abs((acc / R - u * 7).mean()) < 0.01
+
+
+def test_negative_zero_has_sign_zero(orc):
+    levels = orc.uniform_levels(2)
+    v = np.array([-0.0, 0.0, -1e-30, 1.0, -1.0], np.float32)
+    idx, sg, _ = orc.quantize_layer(v, 1.0, levels, SEED, 0, 0, 0)
+    assert sg.tolist() == [0, 0, 1, 0, 1] and idx[:2].tolist() == [0, 0]
 
 
 def test_zero_norm_gives_zero_message(orc):
