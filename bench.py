@@ -39,6 +39,12 @@ def pick_workload(name: str):
         return W.mlp_workload()
     if name == "transformer_xl_small":
         return W.transformer_xl_workload(num_blocks=2, vocab=8192)
+    if name.startswith("flat:"):                       # flat:<log2 n>:<bits>:<K>:<q>
+        n, b, k, q = (int(x) for x in name.split(":")[1:5])
+        return W.flat_workload(n, b, k, q)
+    if name.startswith("ragged:"):                     # ragged:<bits>:<K>:<q>
+        b, k, q = (int(x) for x in name.split(":")[1:4])
+        return W.ragged_workload(b, k, q)
     raise SystemExit(f"unknown workload {name}")
 
 

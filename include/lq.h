@@ -23,7 +23,7 @@
  *    and its d_m values are contiguous.  grads is [K][D_pad], row-major.  Elements between
  *    layers are padding: never interpreted on input, may be overwritten on output.
  *  - A worker's message is W = lq_plan_packed_words() 32-bit words; packed is [K][W].
- *    Every coordinate becomes one symbol of b+1 bits, symbol = sign * 2^b + level index.
+ *    Every coordinate becomes one symbol of b+1 bits, symbol = 2 * level index + sign.
  *    Layer m starts at word_off_m and is cut into blocks of 1024 coordinates (the last one
  *    zero-padded).  A block is (b+1) planes of 32 words.  Coordinate c of a block belongs to
  *    lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane.  The 32 symbols of a lane

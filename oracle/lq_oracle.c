@@ -148,7 +148,7 @@ double orc_round_up_probability(double u, const float* level, int n, int* tau_ou
  * Fixed-width message layout (Section 3.2: a 32-bit float norm, one sign bit and one
  * integer code per coordinate; Section 7.1 footnote: no entropy code on top).
  * The physical layout is this build's:
- *   every coordinate becomes one symbol of b+1 bits, symbol = sign * 2^b + idx;
+ *   every coordinate becomes one symbol of b+1 bits, symbol = 2 * idx + sign (sign in bit 0);
  *   a layer of d coordinates is cut into blocks of 1024 coordinates (the last one
  *   zero-padded); a block is (b+1) planes of 32 words; coordinate c of a block belongs to
  *   lane (c/4)%32 and has position p = 4*(c/128) + c%4 in that lane; the 32 symbols of a
@@ -175,7 +175,7 @@ void orc_pack_layer(const uint8_t* idx, const uint8_t* sign, int64_t d, int b, u
     for (int64_t i = 0; i < d; ++i) {
         int64_t base; int lane, p;
         locate(i, b, &base, &lane, &p);
-        unsigned symbol = ((unsigned)(sign[i] ? 1 : 0) << b) | idx[i];
+        unsigned symbol = ((unsigned)idx[i] << 1) | (unsigned)(sign[i] ? 1 : 0);
         for (int bit = 0; bit <= b; ++bit) {
             if ((symbol >> bit) & 1u) {
                 int t = p * (b + 1) + bit;           /* position in the lane's bit string */
@@ -195,8 +195,8 @@ void orc_unpack_layer(const uint32_t* words, int64_t d, int b, uint8_t* idx, uin
             int t = p * (b + 1) + bit;
             symbol |= ((words[base + (int64_t)(t / 32) * 32 + lane] >> (t % 32)) & 1u) << bit;
         }
-        idx[i] = (uint8_t)(symbol & ((1u << b) - 1u));
-        sign[i] = (uint8_t)(symbol >> b);
+        idx[i] = (uint8_t)(symbol >> 1);
+        sign[i] = (uint8_t)(symbol & 1u);
     }
 }
 

@@ -12,7 +12,7 @@ namespace lq {
 
 constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
 
-// Adds one worker's decoded block into acc.  `table` holds N * l_j for j < n and -N * l_j after.
+// Adds one worker's decoded block into acc.  `table` holds N * l_j at 2j and -N * l_j at 2j + 1.
 template <int B>
 __device__ __forceinline__ void decode_accumulate(float (&acc)[32], const uint32_t* __restrict__ words,
                                                   const float* __restrict__ table)
@@ -70,8 +70,8 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
             const int kk = i / L.nlevels, j = i - kk * L.nlevels;
             const float mag = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
                                         a.levels[(int64_t)layer * kLevelStride + j]);
-            table[kk][j] = mag;
-            table[kk][L.nlevels + j] = -mag;
+            table[kk][2 * j] = mag;                       // symbol = 2 * idx + sign
+            table[kk][2 * j + 1] = -mag;
         }
         __syncthreads();
         if (active)

@@ -9,7 +9,7 @@
 namespace lq {
 
 constexpr int kBlockCoords = 1024;    // coordinates per message block (32 lanes x 32 positions)
-constexpr int kTileBlocks = 32;       // blocks per tile; the 8 warps of a CTA take them round-robin
+constexpr int kTileBlocks = 32;       // blocks per tile; the warps of a CTA take them round-robin
 constexpr int kWarps = 8;
 constexpr int kThreads = 256;
 constexpr int kLevelStride = 256;     // floats per layer in a level table
@@ -68,7 +68,7 @@ cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
 // Encode-side tables derived from one level table (rebuilt whenever the levels change).
 struct SearchTables {
-    uint2* lut;        // [L][kLutStride]  {4 * tau0, bits of the level inside the bin or +inf}
+    uint2* lut;        // [L][kLutStride]  {8 * tau0, bits of the level inside the bin or +inf}
     float2* ld;        // [L][kMaxLevels]  {l_tau, l_{tau+1} - l_tau}
     int32_t* fast;     // [L]              1 if every histogram bin holds at most one level
 };

@@ -3,41 +3,43 @@
 // with the optional histogram of normalised magnitudes (Algorithm 1 line 4) and the sender-side
 // term of the adaptive step size, sum ||V^_{k,t+1/2} - V^_{k,t-1/2}||^2 (Eq. general_stepsize).
 //
-// Work decomposition: one CTA per (tile, worker); a tile is up to 32 blocks of 1024 coordinates of
-// one layer, taken round-robin by the 8 warps.  A lane owns the 32 coordinates {128 j + 4 lane + e}
-// of a block (row j = one float4 per lane, 512 contiguous bytes per warp).  Rows travel from global
-// memory into a per-warp ring of 8 rows in shared memory with 16-byte asynchronous copies, so a
-// warp always has 4 KB in flight and the values never sit in registers while they wait; every lane
-// reads back only the bytes it copied itself, so the ring needs no barrier.  Per row the lane draws
-// one Philox4x32-10 block (4 uniforms); after 8 rows it holds exactly b+1 words of symbols, which it
-// stores plane by plane (128 contiguous bytes per warp and plane).  No shuffles, ballots or atomics
-// on the main path.
+// Work decomposition: one CTA of 8 warps per (tile, worker); a tile is up to 32 blocks of 1024
+// coordinates of one layer, taken round-robin by the warps.  A lane owns the 32 coordinates
+// {128 j + 4 lane + e} of a block (row j = one float4 per lane, 512 contiguous bytes per warp).  Rows
+// travel from global memory into a per-warp ring of 8 rows in shared memory with 16-byte
+// asynchronous copies, so a warp always has 4 KB in flight and the values never sit in registers
+// while they wait; every lane reads back only the bytes it copied itself, so the ring needs no
+// barrier.  Per row the lane draws one Philox4x32-10 block (4 uniforms); after 8 rows it holds
+// exactly b+1 words of symbols, which it stores plane by plane (128 contiguous bytes per warp and
+// plane).  No shuffles, ballots or atomics on the main path.
 //
 // The level search uses a table over the 386 histogram bins of u (exponent + 4 mantissa bits): each
 // entry names the last level at or below the bin's lower edge and the single level that may lie
 // inside the bin, so tau costs one shared-memory load and one compare.  Layers whose levels are
-// denser than the bins fall back to a binary search.  Levels, gaps and the decoded values of the
-// current and the previous message sit in 4-byte tables (conflict-free up to 32 entries); all table
-// offsets are kept pre-scaled by 4.
+// denser than the bins fall back to a binary search.  {level, gap} pairs and the decoded values of the current and the previous message
+// sit in small tables; every table offset derives from one register (8 * tau, then 4 * symbol with
+// symbol = 2 * idx + sign).
 //
-// A row whose 128 values are all +0 (untouched embedding rows, zeroed layers) skips the random
-// numbers and the search: its symbols are 0.  If the previous message is all zero there as well,
-// the row adds nothing to the statistic and is skipped entirely.
+// A row whose 128 values are all zero (untouched embedding rows) skips the random numbers and the
+// search: its symbols are 0.  If the previous message is all zero there as well, the row adds
+// nothing to the statistic and is skipped entirely.
 #include "lq_internal.cuh"
 
 namespace lq {
 
+constexpr int kQWarps = kWarps;                    // warps per CTA of the quantize kernel
+constexpr int kQThreads = kQWarps * 32;
 constexpr int kRingRows = 8;                       // rows of 512 bytes in flight per warp
-constexpr int kRingBytes = kWarps * kRingRows * 512;
+constexpr int kRingBytes = kQWarps * kRingRows * 512;
 
 struct QuantSmem {
-    uint2 lut[kLutStride];           // search table of this layer: {4 * tau0, boundary bits}
-    float lev[kMaxLevels];           // l_tau
-    float gap[kMaxLevels];           // l_{tau+1} - l_tau
-    float tcur[2 * kMaxLevels];      // fp32(N_cur * l_j) by symbol, second half negated
+    uint2 lut[kLutStride];           // search table of this layer: {8 * tau0, boundary bits}
+    float2 ld[kMaxLevels];           // {l_tau, l_{tau+1} - l_tau}
+    float lev[kMaxLevels];           // plain levels (binary-search path)
+    float tcur[2 * kMaxLevels];      // fp32(N_cur * l_idx) at 2 * idx, its negative at 2 * idx + 1
     float tprev[2 * kMaxLevels];     // same for the previous message
     uint32_t hist[LQ_HIST_STRIDE];
-    double scratch[kWarps];
+    double scratch[kQWarps];
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes)
@@ -49,6 +51,38 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// x >> K for a constant K.  kMul writes it as the high half of a multiplication, which runs on the
+// multiply-add pipe instead of the integer/logic pipe.
+template <int K, bool kMul>
+__device__ __forceinline__ uint32_t shr(uint32_t x)
+{
+    if (!kMul) return x >> K;
+    uint32_t d;
+    asm("mul.hi.u32 %0, %1, %2;" : "=r"(d) : "r"(x), "r"(1u << (32 - K)));
+    return d;
+}
+#ifndef LQ_MUL_RHO
+#define LQ_MUL_RHO 1
+#endif
+#ifndef LQ_MUL_SIGN
+#define LQ_MUL_SIGN 0
+#endif
+#ifndef LQ_MUL_LUT
+#define LQ_MUL_LUT 0
+#endif
+
+// x + 8 when a >= b (resp. a < b), else x: one compare and one predicated add
+__device__ __forceinline__ uint32_t add8_if_ge(uint32_t x, float a, float b)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(x) : "f"(a), "f"(b));
+    return x;
+}
+__device__ __forceinline__ uint32_t add8_if_lt(uint32_t x, float a, float b)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(x) : "f"(a), "f"(b));
+    return x;
+}
+
 template <int C>
 __device__ __forceinline__ void put_symbol4(uint32_t (&w)[C], int p, uint32_t sym4)
 {
@@ -57,28 +91,88 @@ __device__ __forceinline__ void put_symbol4(uint32_t (&w)[C], int p, uint32_t sy
     if (s + C > 32) w[i + 1] = sym4 >> (34 - s);
 }
 
+// Philox4x32-10 with counter (c0, layer, worker, step): within one CTA only c0 changes, so half of
+// round 0 (the product with the worker word) and half of round 1 (the product with a word that
+// depends only on round 0's constant half) are the same for every call and are computed once.
+struct PhiloxConsts {
+    uint32_t b;      // step ^ k1                       (round 0: c2' = hi(M0 c0) ^ b)
+    uint32_t c1;     // lo(M1 worker) ^ (k0 + W0)       (round 1: c0'' = hi(M1 c2') ^ c1)
+    uint32_t c2;     // hi(M0 a0) ^ (k1 + W1)           (round 1: c2'' = lo(M0 c0) ^ c2)
+    uint32_t l0;     // lo(M0 a0)                       (round 1: c3'')
+    uint32_t rk0[8], rk1[8];   // the keys of rounds 2..9
+};
+
+__device__ __forceinline__ PhiloxConsts philox_fold(uint32_t layer, uint32_t worker, uint32_t step,
+                                                    uint32_t k0, uint32_t k1)
+{
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * worker;
+    const uint32_t a0 = (uint32_t)(p1 >> 32) ^ layer ^ k0;            // round 0's c0'
+    const uint64_t q0 = (uint64_t)0xD2511F53u * a0;
+    PhiloxConsts pc;
+    pc.b = step ^ k1;
+    pc.c1 = (uint32_t)p1 ^ (k0 + 0x9E3779B9u);
+    pc.c2 = (uint32_t)(q0 >> 32) ^ (k1 + 0xBB67AE85u);
+    pc.l0 = (uint32_t)q0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        pc.rk0[r] = k0 + (uint32_t)(r + 2) * 0x9E3779B9u;
+        pc.rk1[r] = k1 + (uint32_t)(r + 2) * 0xBB67AE85u;
+    }
+    return pc;
+}
+
+__device__ __forceinline__ void philox4x32_10_folded(uint32_t ctr0, const PhiloxConsts& pc, uint32_t (&out)[4])
+{
+    // rounds 0 and 1 with their constant halves folded
+    const uint64_t p0 = (uint64_t)0xD2511F53u * ctr0;
+    const uint32_t c2a = (uint32_t)(p0 >> 32) ^ pc.b;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2a;
+    uint32_t c0 = (uint32_t)(p1 >> 32) ^ pc.c1;
+    uint32_t c1 = (uint32_t)p1;
+    uint32_t c2 = (uint32_t)p0 ^ pc.c2;
+    uint32_t c3 = pc.l0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        const uint64_t q0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t q1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(q1 >> 32) ^ c1 ^ pc.rk0[r];
+        const uint32_t n2 = (uint32_t)(q0 >> 32) ^ c3 ^ pc.rk1[r];
+        c1 = (uint32_t)q1;
+        c3 = (uint32_t)q0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
 // Everything a warp needs to walk its blocks of one (tile, worker).
 struct WarpCtx {
     const float* g;              // first coordinate of the layer in this worker's row
     int64_t size;                // d_m
     uint32_t ring;               // shared-memory address of this lane's 16 bytes in ring row 0
     const float4* ring_ptr;      // the same place as a pointer
-    float r;                     // 1/N, or 0 for a zeroed layer
+    float r;                     // 1/N (zeroed layers, r = 0, take another path)
     int lane;
 };
 
-// Starts the copy of row j of block `blk` into ring row j (zero-filled past the layer's end).
-__device__ __forceinline__ void issue_row(const WarpCtx& c, int64_t blk, int j)
+// Starts the copies of all 8 rows of a block that may reach past the layer's end (zero-filled there).
+__device__ __forceinline__ void issue_ragged_block(const WarpCtx& c, int64_t blk)
 {
-    const int64_t pos = blk * kBlockCoords + 128 * j + 4 * c.lane;
-    const int64_t rem = c.size - pos;
-    const int bytes = rem >= 4 ? 16 : (rem > 0 ? 4 * (int)rem : 0);
-    cp_async16(c.ring + 512u * j, rem > 0 ? c.g + pos : c.g, bytes);
+#pragma unroll
+    for (int j = 0; j < kRingRows; ++j) {
+        const int64_t pos = blk * kBlockCoords + 128 * j + 4 * c.lane;
+        const int64_t rem = c.size - pos;
+        const int bytes = rem >= 4 ? 16 : (rem > 0 ? 4 * (int)rem : 0);
+        cp_async16(c.ring + 512u * j, rem > 0 ? c.g + pos : c.g, bytes);
+        cp_async_commit();
+    }
 }
 
+// One block of 1024 coordinates from the ring.  `next` is this lane's first float4 of the block whose
+// rows replace the consumed ones (nullptr: nothing to fetch).  Returns this lane's statistic term.
 template <int B, bool kFast, bool kHist>
-__device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx& c, int layer, int k,
-                                                 int64_t blk, bool has_next, uint32_t step,
+__device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const WarpCtx& c,
+                                                 int64_t blk, const float* __restrict__ next,
                                                  uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
                                                  bool prev_live, QuantSmem& sm)
 {
@@ -90,29 +184,24 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx
     for (int w = 0; w < C; ++w) cw[w] = 0u;
 
     const char* lut_b = reinterpret_cast<const char*>(sm.lut) - (kLutClamp >> 16);
-    const char* lev_b = reinterpret_cast<const char*>(sm.lev);
-    const char* gap_b = reinterpret_cast<const char*>(sm.gap);
+    const char* ld_b = reinterpret_cast<const char*>(sm.ld);
     const char* tcur_b = reinterpret_cast<const char*>(sm.tcur);
     const char* tprev_b = reinterpret_cast<const char*>(sm.tprev);
     double stat = 0.0;
+    const uint32_t ctr0 = (uint32_t)(blk * 256) + (uint32_t)lane;     // index / 4 of this lane's row 0
 
 #pragma unroll
     for (int j = 0; j < kRingRows; ++j) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r != 0.0f) {
-            cp_async_wait<kRingRows - 1>();
-            v = c.ring_ptr[32 * j];
-            // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
-            v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
-            v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
-        }
+        cp_async_wait<kRingRows - 1>();
+        float4 v = c.ring_ptr[32 * j];
+        // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
+        v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
+        v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
         const float vv[4] = {v.x, v.y, v.z, v.w};
-        const uint32_t any_bits = __float_as_uint(v.x) | __float_as_uint(v.y) | __float_as_uint(v.z) |
-                                  __float_as_uint(v.w);
-        if (kHist || __any_sync(0xffffffffu, any_bits != 0u)) {
+        const float mag = (fabsf(v.x) + fabsf(v.y)) + (fabsf(v.z) + fabsf(v.w));   // 0 iff all four are 0
+        if (kHist || __any_sync(0xffffffffu, mag != 0.0f)) {
             uint32_t x[4];
-            philox4x32_10((uint32_t)(blk * 256 + 32 * j + lane), (uint32_t)layer, (uint32_t)k, step,
-                          p.seed_lo, p.seed_hi, x);
+            philox4x32_10_folded(ctr0 + 32 * j, pc, x);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int pp = 4 * j + e;
@@ -121,11 +210,11 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx
                 // such a u behaves exactly like u = 1 below, so the min(u, 1) of the definition is not needed
                 const float u = __fmul_rn(fabsf(vv[e]), r);
                 const uint32_t ub = __float_as_uint(u);
-                uint32_t t4;
+                uint32_t t8;
                 if (kFast) {
-                    const uint32_t off = (max(ub, kLutClamp) >> 16) & ~7u;
+                    const uint32_t off = shr<16, LQ_MUL_LUT>(max(ub, kLutClamp)) & ~7u;
                     const uint2 en = *reinterpret_cast<const uint2*>(lut_b + off);
-                    t4 = en.x + (u >= __uint_as_float(en.y) ? 4u : 0u);
+                    t8 = add8_if_ge(en.x, u, __uint_as_float(en.y));
                 } else {
                     int tau = 0;
 #pragma unroll
@@ -133,23 +222,22 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx
                         const int cand = tau + (1 << s);
                         if (sm.lev[cand] <= u) tau = cand;
                     }
-                    t4 = 4u * (uint32_t)min(tau, n - 2);
+                    t8 = 8u * (uint32_t)min(tau, n - 2);
                 }
-                const float l0 = *reinterpret_cast<const float*>(lev_b + t4);
-                const float den = *reinterpret_cast<const float*>(gap_b + t4);
-                const float num = __fsub_rn(u, l0);
+                const float2 ld = *reinterpret_cast<const float2*>(ld_b + t8);
+                const float den = ld.y;
+                const float num = __fsub_rn(u, ld.x);
                 // rho = (x >> 9) * 2^-23; f = 1 + rho is built from the bits, and fma(f, den, -den)
                 // rounds the exact product rho * den once, like the plain multiplication
-                const float f = __uint_as_float(__funnelshift_r(x[e], 0x7Fu, 9));
+                const float f = __uint_as_float(shr<9, LQ_MUL_RHO>(x[e]) + 0x3F800000u);
                 const float t = __fmaf_rn(f, den, -den);
-                const uint32_t i4 = t4 + (t < num ? 4u : 0u);
-                const uint32_t sym4 = i4 | ((bits >> (29 - B)) & (4u * n));
+                const uint32_t i8 = add8_if_lt(t8, t, num);
+                const uint32_t sym4 = i8 | (shr<29, LQ_MUL_SIGN>(bits) & 4u);     // 4 * (2 * idx + sign)
                 put_symbol4<C>(cw, pp, sym4);
 
                 if (kHist) {
                     const int64_t pos = blk * kBlockCoords + 128 * j + 4 * lane + e;
-                    if (r != 0.0f && pos < c.size)
-                        atomicAdd(&sm.hist[(max(ub, kLutClamp) - kLutClamp) >> 19], 1u);
+                    if (pos < c.size) atomicAdd(&sm.hist[(max(ub, kLutClamp) - kLutClamp) >> 19], 1u);
                 }
 
                 // step-size statistic: fp32 difference of the two decoded values, squared in fp64
@@ -162,14 +250,12 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, 4 * j + e));
-                const double dd = (double)__fsub_rn(0.0f, prv);
+                const double dd = (double)prv;
                 stat = fma(dd, dd, stat);
             }
         }
-        if (r != 0.0f) {
-            if (has_next) issue_row(c, blk + kWarps, j);
-            cp_async_commit();
-        }
+        if (next) cp_async16(c.ring + 512u * j, next + 128 * j, 16);
+        cp_async_commit();
     }
     const int64_t woff = blk * (int64_t)C * 32 + lane;
 #pragma unroll
@@ -177,9 +263,34 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const WarpCtx
     return stat;
 }
 
+// A layer whose message is all zero (zero norm, NaN or Inf inside): zero words, and the statistic is
+// the squared previous message.
+template <int B>
+__device__ __forceinline__ double zeroed_tile(const Tile& tile, int lane, uint32_t* __restrict__ out,
+                                              const uint32_t* __restrict__ prev, QuantSmem& sm)
+{
+    constexpr int C = B + 1;
+    double stat = 0.0;
+    for (int b = threadIdx.x >> 5; b < tile.nblocks; b += kQWarps) {
+        const int64_t woff = (tile.block0 + b) * (int64_t)C * 32 + lane;
+        uint32_t pw[C];
+#pragma unroll
+        for (int w = 0; w < C; ++w) {
+            pw[w] = prev ? __ldcs(prev + woff + w * 32) : 0u;
+            __stcs(out + woff + w * 32, 0u);
+        }
+#pragma unroll
+        for (int pp = 0; pp < 32; ++pp) {
+            const double dd = (double)sm.tprev[symbol4_at<C>(pw, pp) >> 2];
+            stat = fma(dd, dd, stat);
+        }
+    }
+    return stat;
+}
+
 template <int B, bool kFast, bool kHist>
-__device__ __forceinline__ double quantize_tile(const PlanDev& p, const WarpCtx& c, const Tile& tile, int layer,
-                                                int k, uint32_t step, uint32_t* __restrict__ out,
+__device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const WarpCtx& c, const Tile& tile,
+                                                uint32_t* __restrict__ out,
                                                 const uint32_t* __restrict__ prev, QuantSmem& sm)
 {
     constexpr int C = B + 1;
@@ -188,24 +299,31 @@ __device__ __forceinline__ double quantize_tile(const PlanDev& p, const WarpCtx&
     if (warp >= tile.nblocks) return stat;
     int64_t blk = tile.block0 + warp;
     const int64_t end = tile.block0 + tile.nblocks;
-    if (c.r != 0.0f) {
+    const int64_t nfull = c.size / kBlockCoords;          // blocks below this index lie inside the layer
+    if (blk < nfull) {
+        const float* src = c.g + blk * kBlockCoords + 4 * c.lane;
 #pragma unroll
-        for (int j = 0; j < kRingRows; ++j) { issue_row(c, blk, j); cp_async_commit(); }
+        for (int j = 0; j < kRingRows; ++j) { cp_async16(c.ring + 512u * j, src + 128 * j, 16); cp_async_commit(); }
+    } else {
+        issue_ragged_block(c, blk);
     }
     uint32_t pw[C];
 #pragma unroll
     for (int w = 0; w < C; ++w) pw[w] = prev ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
-    for (; blk < end; blk += kWarps) {
-        const bool has_next = blk + kWarps < end;
+    for (; blk < end; blk += kQWarps) {
+        const int64_t nblk = blk + kQWarps;
+        const bool has_next = nblk < end;
         uint32_t pn[C];                                   // the next block's previous words, fetched early
 #pragma unroll
         for (int w = 0; w < C; ++w)
-            pn[w] = (prev && has_next) ? __ldcs(prev + (blk + kWarps) * (int64_t)C * 32 + c.lane + w * 32) : 0u;
+            pn[w] = (prev && has_next) ? __ldcs(prev + nblk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
         uint32_t por = 0u;
 #pragma unroll
         for (int w = 0; w < C; ++w) por |= pw[w];
         const bool prev_live = __any_sync(0xffffffffu, por != 0u);
-        stat += quantize_block<B, kFast, kHist>(p, c, layer, k, blk, has_next, step, out, pw, prev_live, sm);
+        const float* next = (has_next && nblk < nfull) ? c.g + nblk * kBlockCoords + 4 * c.lane : nullptr;
+        stat += quantize_block<B, kFast, kHist>(pc, c, blk, next, out, pw, prev_live, sm);
+        if (has_next && nblk >= nfull) issue_ragged_block(c, nblk);   // the layer's last, partial block
 #pragma unroll
         for (int w = 0; w < C; ++w) pw[w] = pn[w];
     }
@@ -214,7 +332,7 @@ __device__ __forceinline__ double quantize_tile(const PlanDev& p, const WarpCtx&
 }
 
 template <bool kHist>
-__global__ void __launch_bounds__(kThreads, 3) quantize_pack_kernel(
+__global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     PlanDev p, const float* __restrict__ grads, uint32_t step, uint32_t* __restrict__ packed,
     const float* __restrict__ norms, uint32_t* __restrict__ hist,
     const uint32_t* __restrict__ prev_packed, const float* __restrict__ prev_norms,
@@ -237,11 +355,10 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_pack_kernel(
         const float l = levels_cur[(int64_t)layer * kLevelStride + i];
         const float c = __fmul_rn(ncur, l);
         const float q = __fmul_rn(nprev, levels_prev[(int64_t)layer * kLevelStride + i]);
-        const float2 ld = st.ld[(int64_t)layer * kMaxLevels + i];
-        sm.lev[i] = fast ? ld.x : l;                  // the binary search reads plain levels, all n of them
-        sm.gap[i] = ld.y;
-        sm.tcur[i] = c;  sm.tcur[n + i] = -c;
-        sm.tprev[i] = q; sm.tprev[n + i] = -q;
+        sm.ld[i] = st.ld[(int64_t)layer * kMaxLevels + i];
+        sm.lev[i] = l;
+        sm.tcur[2 * i] = c;  sm.tcur[2 * i + 1] = -c;
+        sm.tprev[2 * i] = q; sm.tprev[2 * i + 1] = -q;
     }
     if (fast)
         for (int i = threadIdx.x; i < LQ_NUM_BINS; i += blockDim.x)
@@ -257,14 +374,17 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_pack_kernel(
     c.ring = (uint32_t)__cvta_generic_to_shared(c.ring_ptr);
     c.r = p.rnorm[kl];
     c.lane = lane;
+    const bool zeroed = c.r == 0.0f;
+    const PhiloxConsts pc = philox_fold((uint32_t)layer, (uint32_t)k, step, p.seed_lo, p.seed_hi);
     uint32_t* out = packed + (int64_t)k * p.packed_words + L.word_off;
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
 
     double stat = 0.0;
-    switch (L.bits * 2 + (fast ? 1 : 0)) {
+    switch (zeroed ? -L.bits : L.bits * 2 + (fast ? 1 : 0)) {
 #define LQ_CASE(BB)                                                                                   \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(p, c, tile, layer, k, step, out, prev, sm); break; \
-    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(p, c, tile, layer, k, step, out, prev, sm); break;
+    case -BB:        stat = zeroed_tile<BB>(tile, lane, out, prev, sm); break;                        \
+    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(pc, c, tile, out, prev, sm); break; \
+    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(pc, c, tile, out, prev, sm); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
@@ -295,7 +415,7 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 
 // One CTA per layer: derives the encode-side tables from the layer's levels.
 //   ld[tau]  = {l_tau, l_{tau+1} - l_tau}                 tau = 0..n-2 (other entries: {l_tau, 0})
-//   lut[bin] = {4 * tau0, bits of l_{tau0+1} if it lies inside the bin, else +inf}
+//   lut[bin] = {8 * tau0, bits of l_{tau0+1} if it lies inside the bin, else +inf}
 //              tau0 = last level (<= n-2) at or below the bin's lower edge
 //   fast     = no bin holds two or more levels (then tau is tau0 or tau0 + 1)
 __global__ void __launch_bounds__(128) build_search_kernel(PlanDev p, const float* __restrict__ levels,
@@ -323,7 +443,7 @@ __global__ void __launch_bounds__(128) build_search_kernel(PlanDev p, const floa
             boundary = __float_as_uint(lev[tau0 + 1]);
             if (tau0 + 2 <= n - 2 && lev[tau0 + 2] < hi) atomicOr(&slow, 1);
         }
-        t.lut[(int64_t)m * kLutStride + bin] = make_uint2(4u * (uint32_t)tau0, boundary);
+        t.lut[(int64_t)m * kLutStride + bin] = make_uint2(8u * (uint32_t)tau0, boundary);
     }
     __syncthreads();
     if (threadIdx.x == 0) t.fast[m] = slow ? 0 : 1;
@@ -344,11 +464,11 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
     if (p.num_tiles == 0) return cudaSuccess;
     const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
     if (hist)
-        quantize_pack_kernel<true><<<grid, kThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist, prev_packed,
-                                                             prev_norms, levels_cur, levels_prev, t);
+        quantize_pack_kernel<true><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist,
+                                                                         prev_packed, prev_norms, levels_cur, levels_prev, t);
     else
-        quantize_pack_kernel<false><<<grid, kThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist, prev_packed,
-                                                              prev_norms, levels_cur, levels_prev, t);
+        quantize_pack_kernel<false><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist,
+                                                                          prev_packed, prev_norms, levels_cur, levels_prev, t);
     return cudaGetLastError();
 }
 

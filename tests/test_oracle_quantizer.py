@@ -241,36 +241,40 @@ def test_pack_roundtrip_all_widths_and_tails(orc):
 
 def test_pack_layout_hand_worked_positions(orc):
     """Positions worked out by hand from the layout text: block of 1024 coordinates, lane
-    (c/4)%32, position p = 4*(c/128) + c%4, symbol = sign*2^b + idx of b+1 bits at bit offset
+    (c/4)%32, position p = 4*(c/128) + c%4, symbol = 2*idx + sign of b+1 bits at bit offset
     p*(b+1) of the lane's string, bit t in word (t/32)*32 + lane."""
     b = 3                                      # 4-bit symbols, 4 planes of 32 words per block
     d = 1200
     for (i, code, expect) in [
-        # i = 0: block 0, lane 0, p 0 -> symbol 1101 in bits 0..3 of word 0
-        (0, 0b101, {0: 0b1101}),
+        # i = 0: block 0, lane 0, p 0 -> symbol 101|1 = 1011 in bits 0..3 of word 0
+        (0, 0b101, {0: 0b1011}),
         # i = 129: c = 129, lane 32%32 = 0, p = 4*1+1 = 5 -> bits 20..23 of word 0
         (129, 0b111, {0: 0b1111 << 20}),
-        # i = 7: lane 1, p = 3 -> bits 12..15 of word 1
-        (7, 0b010, {1: 0b1010 << 12}),
-        # i = 1023: lane 31, p = 31 -> bits 124..127 -> plane 3 (word 96+31) bits 28..31
-        (1023, 0b110, {96 + 31: 0b1110 << 28}),
-        # i = 427: lane 106%32 = 10, p = 4*3+3 = 15 -> bits 60..63 -> plane 1 (word 32+10) bits 28..31
-        (427, 0b011, {32 + 10: 0b1011 << 28}),
-        # second block: i = 1028 -> block base 128 words, lane 1, p 0
-        (1028, 0b001, {128 + 1: 0b1001}),
+        # i = 7: lane 1, p = 3 -> bits 12..15 of word 1; symbol 010|1 = 0101
+        (7, 0b010, {1: 0b0101 << 12}),
+        # i = 1023: lane 31, p = 31 -> bits 124..127 -> plane 3 (word 96+31) bits 28..31; symbol 110|1
+        (1023, 0b110, {96 + 31: 0b1101 << 28}),
+        # i = 427: lane 106%32 = 10, p = 4*3+3 = 15 -> bits 60..63 -> plane 1 (word 32+10) bits 28..31; 011|1
+        (427, 0b011, {32 + 10: 0b0111 << 28}),
+        # second block: i = 1028 -> block base 128 words, lane 1, p 0; symbol 001|1
+        (1028, 0b001, {128 + 1: 0b0011}),
     ]:
         idx = np.zeros(d, np.uint8); sg = np.zeros(d, np.uint8)
         idx[i] = code; sg[i] = 1
         w = orc.pack_layer(idx, sg, b)
         got = {int(j): int(w[j]) for j in np.flatnonzero(w)}
         assert got == expect, (i, got, expect)
+    # a positive coordinate leaves bit 0 of its symbol clear: i = 4 (lane 1, p 0), idx 6 -> 1100
+    idx = np.zeros(d, np.uint8); sg = np.zeros(d, np.uint8); idx[4] = 6
+    w = orc.pack_layer(idx, sg, b)
+    assert {int(j): int(w[j]) for j in np.flatnonzero(w)} == {1: 0b1100}
     # b = 4: 5-bit symbols straddle words; p = 6 (i = 128 + 4*lane + 2, lane 3 -> i = 142) sits at
     # bits 30..34: two bits in plane 0 and three in plane 1
     idx = np.zeros(200, np.uint8); sg = np.zeros(200, np.uint8)
-    idx[142] = 0b1011; sg[142] = 1                  # symbol 11011
+    idx[142] = 0b1011; sg[142] = 1                  # symbol 1011|1 = 10111
     w = orc.pack_layer(idx, sg, 4)
     got = {int(j): int(w[j]) for j in np.flatnonzero(w)}
-    assert got == {3: 0b11 << 30, 32 + 3: 0b110}
+    assert got == {3: 0b11 << 30, 32 + 3: 0b101}
 
 
 # ---------------------------------------------------------------------------- histogram
