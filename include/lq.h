@@ -149,6 +149,25 @@ int qoda_get_scalars(const lq_plan* plan, int64_t* t, double* S, double* eta);
  * last norm computation.  Either may be NULL.  Synchronises. */
 int lq_get_statistics(const lq_plan* plan, double* host_sq_diff, uint32_t* host_flags);
 
+/* L^q norm of one device vector with no allocation anywhere (the paper has no counterpart: this is
+ * a convenience of the library).  For callers that cannot allocate device memory when they need a
+ * norm - all device memory already belongs to another allocator, or the device-wide
+ * synchronisation that cudaMalloc and cudaFree imply is not acceptable where the call sits - and
+ * who therefore cannot create a plan.  The scratch of the two-stage reduction is a fixed array
+ * inside the library image (32 KB on every GPU that loads the library, held until the process
+ * exits), so this call and everything below it call no cudaMalloc, cudaFree or allocating routine.
+ *   v dev [n] fp32, 16-byte aligned (may be NULL when n = 0);  n in [0, 134217728] (4096 tiles of
+ *   32768 values: larger n is refused with LQ_EINVAL);  q as in lq_plan_create (0 = infinity
+ *   norm, 1..16);  norm_out dev [1]: fp32(||v||_q) accumulated in fp64, or 0 when flagged;
+ *   status_out dev [1] or NULL: 0, LQ_STATUS_ZERO_NORM or LQ_STATUS_NONFINITE.
+ * Asynchronous on `stream`.  The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, which may load the module on that device); make that first call before
+ * any stream capture begins.  All calls share the one array and every call overwrites the
+ * entries it reads back, so nothing needs clearing, but calls that overlap on the GPU (two
+ * streams, two host threads) race on it: order them. */
+int lq_vector_norm_static(const float* v, int64_t n, int32_t q, float* norm_out, uint32_t* status_out,
+                          void* stream);
+
 /* Measurement aid (no counterpart in the paper).  While enabled, every kernel the library
  * launches for this plan is bracketed by two CUDA events on the caller's stream.
  * lq_profile_read synchronises the device, returns per kernel the summed device time in

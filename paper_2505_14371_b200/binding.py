@@ -24,7 +24,8 @@ STATUS_NONFINITE = 2
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "lq_get_statistics", "lq_profile_enable", "lq_profile_read",
+           "qoda_get_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
+           "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
                 "decode", "fit"]
@@ -62,6 +63,7 @@ def load_library() -> C.CDLL:
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
+    L.lq_vector_norm_static.argtypes = [vp, i64, i32, vp, vp, vp]
     L.lq_profile_enable.argtypes = [vp, i32]
     L.lq_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
     L.lq_error_string.argtypes = [C.c_int]; L.lq_error_string.restype = C.c_char_p
@@ -90,6 +92,17 @@ def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
 
 def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
+
+
+def lq_vector_norm_static(v: torch.Tensor, q: int, norm_out: torch.Tensor,
+                          status_out: Optional[torch.Tensor] = None) -> None:
+    """L^q norm of the fp32 device vector `v` into norm_out[0] through the library's fixed scratch
+    array: no plan and no allocation below this call.  For callers whose device memory is all
+    spoken for, or who cannot afford the synchronisation an allocation implies.  Calls must not
+    overlap on the GPU (they share the scratch)."""
+    _check(load_library().lq_vector_norm_static(_ptr(v, torch.float32), v.numel(), int(q),
+                                                _ptr(norm_out, torch.float32), _ptr(status_out, torch.int32),
+                                                _stream()))
 
 
 class Plan:

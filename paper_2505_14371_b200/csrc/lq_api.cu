@@ -25,6 +25,20 @@ int fail(int code, const char* fmt, ...)
     return code;
 }
 
+}  // namespace
+
+// Records a failure reason for lq_last_error() from another translation unit of the library.
+int lq::lq_set_error(int code, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+namespace {
+
 #define LQ_CUDA(expr)                                                                         \
     do {                                                                                      \
         cudaError_t e_ = (expr);                                                              \

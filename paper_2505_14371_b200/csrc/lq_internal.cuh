@@ -63,6 +63,9 @@ struct PlanDev {
     QodaScalars* scalars;
 };
 
+// Stores a printf-style reason for lq_last_error() (calling thread) and returns `code`.
+int lq_set_error(int code, const char* fmt, ...);
+
 // ---- launchers (each enqueues on `s` and returns the launch status) ----
 cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream_t s);
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
