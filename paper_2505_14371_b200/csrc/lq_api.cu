@@ -68,6 +68,8 @@ struct lq_plan {
     bool have_message = false;
     bool qoda_ready = false;
     bool stat_pending = false;
+    uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
+    int mask_cur = 0;
     // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
     struct ProfRec { int id; cudaEvent_t a, b; };
     bool profiling = false;
@@ -84,7 +86,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -152,7 +154,15 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
 
     lq_plan* p = new (std::nothrow) lq_plan;
     if (!p) return fail(LQ_ENOMEM, "host allocation failed");
-    int64_t elem = 0, word = 0, ntiles = 0;
+    int64_t elem = 0, word = 0, ntiles = 0, blocks = 0;
+    // tile size: as large as possible while (tiles x workers) still fills the GPU several times over
+    int tile_blocks = kTileBlocks;
+    {
+        int64_t total = 0;
+        for (int m = 0; m < num_layers; ++m)
+            if (layer_sizes[m] > 0) total += (layer_sizes[m] + kBlockCoords - 1) / kBlockCoords;
+        while (tile_blocks > kSubBlocks && (total / tile_blocks) * num_workers < 4096) tile_blocks /= 2;
+    }
     try {
         p->layers.resize((size_t)num_layers);
         for (int m = 0; m < num_layers; ++m) {
@@ -164,17 +174,19 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
             L.elem_off = elem; L.word_off = word; L.size = d; L.bits = b; L.nlevels = 1 << b;
             L.nblocks = (int32_t)((d + kBlockCoords - 1) / kBlockCoords);
             L.first_tile = (int32_t)ntiles;
-            L.ntiles = (L.nblocks + kTileBlocks - 1) / kTileBlocks;
+            L.ntiles = (L.nblocks + tile_blocks - 1) / tile_blocks;
             L.pad_ = 0;
+            L.block_off = blocks;
+            blocks += L.nblocks;
             for (int t = 0; t < L.ntiles; ++t) {
                 Tile tl;
-                tl.layer = m; tl.block0 = t * kTileBlocks;
-                tl.nblocks = L.nblocks - tl.block0 < kTileBlocks ? L.nblocks - tl.block0 : kTileBlocks;
+                tl.layer = m; tl.block0 = t * tile_blocks;
+                tl.nblocks = L.nblocks - tl.block0 < tile_blocks ? L.nblocks - tl.block0 : tile_blocks;
                 tl.pad_ = 0;
                 p->tiles.push_back(tl);
             }
             ntiles += L.ntiles;
-            if (ntiles >= ((int64_t)1 << 31) - 1) { delete p; return fail(LQ_EINVAL, "too many tiles"); }
+            if (ntiles >= ((int64_t)1 << 29)) { delete p; return fail(LQ_EINVAL, "too many tiles"); }
             elem += (d + 31) / 32 * 32;
             word += (int64_t)L.nblocks * 32 * (b + 1);
         }
@@ -186,7 +198,8 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     p->seed = seed;
     PlanDev& d = p->dev;
     d.num_layers = num_layers; d.num_tiles = (int32_t)ntiles; d.num_workers = num_workers; d.q = q;
-    d.padded_elems = elem; d.packed_words = word;
+    d.sub_tiles = tile_blocks / kSubBlocks;
+    d.padded_elems = elem; d.packed_words = word; d.total_blocks = blocks;
     d.seed_lo = (uint32_t)seed; d.seed_hi = (uint32_t)(seed >> 32);
 
     cudaError_t e = cudaGetDevice(&p->device);
@@ -202,11 +215,14 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.lut, nl * kLutStride);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.ld, nl * kMaxLevels);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.fast, nl);
-    if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT * (size_t)d.sub_tiles);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.stat_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
+    for (int i = 0; i < 2; ++i)
+        if (e == cudaSuccess) e = dev_alloc_zero(&p->d_row_mask[i], (size_t)num_workers * (size_t)(blocks ? blocks : 1));
+    d.row_mask = p->d_row_mask[0]; d.row_mask_prev = nullptr;
     if (e == cudaSuccess) e = dev_alloc_zero(&d.scalars, 1);
     if (e == cudaSuccess && !p->layers.empty())
         e = cudaMemcpy(p->d_layers, p->layers.data(), p->layers.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice);
@@ -303,7 +319,7 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
     if (plan->dev.num_layers == 0) return LQ_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const PlanDev& d = plan->dev;
-    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, false, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
     return LQ_OK;
 }
@@ -329,10 +345,14 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     } else {
         plan->prev = plan->cur;
     }
+    // the masks written now describe this message; the ones of the last call describe prev_packed
+    plan->dev.row_mask_prev = plan->have_message ? plan->d_row_mask[plan->mask_cur] : nullptr;
+    plan->mask_cur = plan->have_message ? 1 - plan->mask_cur : plan->mask_cur;
+    plan->dev.row_mask = plan->d_row_mask[plan->mask_cur];
     const PlanDev& d = plan->dev;
     const float* lc = plan->d_levels_enc[plan->cur];
     const float* lp = plan->d_levels_enc[plan->prev];
-    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, s); }));
+    LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, true, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_QUANTIZE_PACK, s, [&] {
         return launch_quantize(d, grads, step, packed, norms, hist, prev_packed, prev_norms, lc, lp,

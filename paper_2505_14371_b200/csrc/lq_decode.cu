@@ -1,7 +1,7 @@
 // DECODE + aggregate of the K workers' messages, alone or fused with the optimistic dual averaging
 // update (Algorithm 1 lines 15-18 and line 10 of the next iteration; Eq. ODA; Eq. general_stepsize).
 //
-// One CTA per tile (up to 32 blocks of 1024 coordinates of one layer, taken round-robin by 8 warps).  A lane
+// One CTA per sub-tile (up to 32 blocks of 1024 coordinates of one layer, taken round-robin by 8 warps).  A lane
 // owns the same 32 coordinates it owned at encode time, so it reads (b+1) words per worker with
 // 128-byte coalesced warp loads, looks the signed decoded values up by symbol in a per-(worker, layer) table in shared
 // memory, sums them in worker order in registers, and finishes with float4 reads of Y and X_1 and
@@ -12,19 +12,35 @@ namespace lq {
 
 constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
 
-// Adds one worker's decoded block into acc.  `table` holds N * l_j at 2j and -N * l_j at 2j + 1.
-template <int B>
-__device__ __forceinline__ void decode_accumulate(float (&acc)[32], const uint32_t* __restrict__ words,
-                                                  const float* __restrict__ table)
+
+// Adds up to kWorkerChunk workers' decoded half blocks into acc, in worker order.  Half H of a lane's
+// string holds its symbols 16 H .. 16 H + 15 (rows 4 H .. 4 H + 3 of the block); only the words that
+// carry those symbols are read.  All workers' words are requested before the first one is used, so
+// that a warp keeps a few KB in flight.  `table[kk]` holds N * l_j at 2j and -N * l_j at 2j + 1 for
+// worker kk of the chunk.
+template <int B, int H>
+__device__ __forceinline__ void decode_accumulate(float (&acc)[16], const uint32_t* __restrict__ words,
+                                                  int64_t worker_stride, int kc,
+                                                  const float (*table)[2 * kMaxLevels])
 {
     constexpr int C = B + 1;
-    uint32_t w[C];
+    constexpr int kFirst = (16 * H * C) >> 5;                         // first and last word of this half
+    constexpr int kLast = ((16 * (H + 1) * C) - 1) >> 5;
+    uint32_t w[kWorkerChunk][C];
 #pragma unroll
-    for (int i = 0; i < C; ++i) w[i] = __ldcs(words + i * 32);
-    const char* tb = reinterpret_cast<const char*>(table);
+    for (int kk = 0; kk < kWorkerChunk; ++kk)
 #pragma unroll
-    for (int p = 0; p < 32; ++p)
-        acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w, p));
+        for (int i = 0; i < C; ++i)
+            w[kk][i] = (i >= kFirst && i <= kLast && kk < kc) ? __ldcs(words + kk * worker_stride + i * 32) : 0u;
+#pragma unroll
+    for (int kk = 0; kk < kWorkerChunk; ++kk) {
+        if (kk < kc) {
+            const char* tb = reinterpret_cast<const char*>(table[kk]);
+#pragma unroll
+            for (int p = 0; p < 16; ++p)
+                acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w[kk], 16 * H + p));
+        }
+    }
 }
 
 struct DecodeArgs {
@@ -38,59 +54,54 @@ struct DecodeArgs {
     float* gbar;
 };
 
-// Any worker count: the accumulators live across chunks of kWorkerChunk workers.
-template <int B, bool kQoda>
-__device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
-                                                     const Tile& tile, const DecodeArgs& a,
-                                                     float (*table)[2 * kMaxLevels], float eta)
+// Fills the value tables of workers k0 .. k0 + kc - 1 of one layer (CTA-wide, between two barriers).
+__device__ __forceinline__ void fill_tables(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
+                                            float (*table)[2 * kMaxLevels], int k0, int kc)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int K = p.num_workers;
-    const float invK = __fdiv_rn(1.0f, (float)K);
-    // each warp takes the tile's blocks round-robin; all warps run the same number of rounds so
-    // that the table refills (CTA-wide barriers) stay aligned
-    for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
-    const bool active = b0 + warp < tile.nblocks;
-    const int64_t blk = tile.block0 + b0 + warp;
-    const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
-    float acc[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-
-    for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
-        if (K <= kWorkerChunk && b0 > 0) {          // one chunk only: the table is already in place
-            if (active)
-                for (int kk = 0; kk < K; ++kk)
-                    decode_accumulate<B>(acc, a.packed + (int64_t)kk * p.packed_words + woff, table[kk]);
-            break;
-        }
-        const int kc = min(kWorkerChunk, K - k0);
-        __syncthreads();
-        for (int i = threadIdx.x; i < kc * L.nlevels; i += blockDim.x) {
-            const int kk = i / L.nlevels, j = i - kk * L.nlevels;
-            const float mag = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
-                                        a.levels[(int64_t)layer * kLevelStride + j]);
-            table[kk][2 * j] = mag;                       // symbol = 2 * idx + sign
-            table[kk][2 * j + 1] = -mag;
-        }
-        __syncthreads();
-        if (active)
-            for (int kk = 0; kk < kc; ++kk)
-                decode_accumulate<B>(acc, a.packed + (int64_t)(k0 + kk) * p.packed_words + woff, table[kk]);
+    __syncthreads();
+    for (int i = threadIdx.x; i < kc * L.nlevels; i += blockDim.x) {
+        const int kk = i / L.nlevels, j = i - kk * L.nlevels;
+        const float mag = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
+                                    a.levels[(int64_t)layer * kLevelStride + j]);
+        table[kk][2 * j] = mag;                       // symbol = 2 * idx + sign
+        table[kk][2 * j + 1] = -mag;
     }
-    if (!active) continue;
+    __syncthreads();
+}
+
+// One half block: the mean of the K decoded messages for rows 4 H .. 4 H + 3, then the update.
+// Any worker count: the accumulators live across chunks of kWorkerChunk workers; with a single chunk
+// the tables are filled once per CTA (`resident`).
+template <int B, int H, bool kQoda>
+__device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
+                                            float (*table)[2 * kMaxLevels], float eta, float invK,
+                                            int64_t blk, bool active, bool& resident)
+{
+    const int lane = threadIdx.x & 31;
+    const int K = p.num_workers;
+    const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
+    float acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+    for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
+        const int kc = min(kWorkerChunk, K - k0);
+        if (!resident) fill_tables(p, L, layer, a, table, k0, kc);
+        if (K <= kWorkerChunk) resident = true;
+        if (active) decode_accumulate<B, H>(acc, a.packed + (int64_t)k0 * p.packed_words + woff, p.packed_words, kc, table);
+    }
+    if (!active) return;
 
     const int64_t base = L.elem_off + blk * kBlockCoords + 4 * lane;
     const int64_t limit = L.elem_off + L.size;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int64_t pos = base + 128 * j;
+    for (int jj = 0; jj < 4; ++jj) {
+        const int64_t pos = base + 128 * (4 * H + jj);
         if (pos >= limit) continue;
         float4 g;
-        g.x = __fmul_rn(acc[4 * j + 0], invK);
-        g.y = __fmul_rn(acc[4 * j + 1], invK);
-        g.z = __fmul_rn(acc[4 * j + 2], invK);
-        g.w = __fmul_rn(acc[4 * j + 3], invK);
+        g.x = __fmul_rn(acc[4 * jj + 0], invK);
+        g.y = __fmul_rn(acc[4 * jj + 1], invK);
+        g.z = __fmul_rn(acc[4 * jj + 2], invK);
+        g.w = __fmul_rn(acc[4 * jj + 3], invK);
         if (a.gbar) *reinterpret_cast<float4*>(a.gbar + pos) = g;
         if (kQoda) {
             const float4 y0 = *reinterpret_cast<const float4*>(a.Y + pos);
@@ -107,14 +118,35 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
             if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
         }
     }
+}
+
+template <int B, bool kQoda>
+__device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
+                                                     const Tile& tile, const DecodeArgs& a,
+                                                     float (*table)[2 * kMaxLevels], float eta)
+{
+    const int warp = threadIdx.x >> 5;
+    const float invK = __fdiv_rn(1.0f, (float)p.num_workers);
+    bool resident = false;
+    // each warp takes the tile's blocks round-robin; all warps run the same number of rounds so
+    // that the table refills (CTA-wide barriers) stay aligned
+    for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
+        const bool active = b0 + warp < tile.nblocks;
+        const int64_t blk = tile.block0 + b0 + warp;
+        decode_half<B, 0, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident);
+        decode_half<B, 1, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident);
     }
 }
 
 template <bool kQoda>
-__global__ void __launch_bounds__(kThreads) decode_kernel(PlanDev p, DecodeArgs a)
+__global__ void __launch_bounds__(kThreads, 4) decode_kernel(PlanDev p, DecodeArgs a)
 {
     __shared__ float table[kWorkerChunk][2 * kMaxLevels];
-    const Tile tile = p.tiles[blockIdx.x];
+    Tile tile = p.tiles[blockIdx.x / p.sub_tiles];                    // this CTA takes one sub-tile of it
+    const int sub0 = (blockIdx.x % p.sub_tiles) * kSubBlocks;
+    if (sub0 >= tile.nblocks) return;
+    tile.block0 += sub0;
+    tile.nblocks = min(kSubBlocks, tile.nblocks - sub0);
     const int layer = tile.layer;
     const LayerDesc L = p.layers[layer];
     const float eta = kQoda ? p.scalars->eta : 0.0f;
@@ -168,8 +200,8 @@ cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float*
 {
     if (p.num_tiles == 0) return cudaSuccess;
     DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
-    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles, kThreads, 0, s>>>(p, a);
-    else      decode_kernel<false><<<(unsigned)p.num_tiles, kThreads, 0, s>>>(p, a);
+    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, 0, s>>>(p, a);
+    else      decode_kernel<false><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, 0, s>>>(p, a);
     return cudaGetLastError();
 }
 

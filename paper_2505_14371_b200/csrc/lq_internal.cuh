@@ -9,7 +9,9 @@
 namespace lq {
 
 constexpr int kBlockCoords = 1024;    // coordinates per message block (32 lanes x 32 positions)
-constexpr int kTileBlocks = 32;       // blocks per tile; the warps of a CTA take them round-robin
+constexpr int kTileBlocks = 128;      // most blocks per tile (the encoder's unit: its per-CTA tables are amortised over a
+                                      // tile); a plan uses 32, 64 or 128, the largest that still gives several waves of CTAs
+constexpr int kSubBlocks = 32;        // blocks per sub-tile (the unit of the norm and decode kernels)
 constexpr int kWarps = 8;
 constexpr int kThreads = 256;
 constexpr int kLevelStride = 256;     // floats per layer in a level table
@@ -27,6 +29,7 @@ struct LayerDesc {
     int32_t first_tile;   // tiles of one layer are contiguous in the tile table
     int32_t ntiles;
     int32_t pad_;
+    int64_t block_off;    // first block of the layer in a worker's row of the zero-row masks
 };
 
 struct Tile {
@@ -52,14 +55,18 @@ struct PlanDev {
     int32_t num_tiles;
     int32_t num_workers;
     int32_t q;            // 0 = infinity norm
+    int32_t sub_tiles;    // sub-tiles per tile: the plan's tile size / kSubBlocks
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;
-    double* norm_partial; // [K][num_tiles]
+    double* norm_partial; // [K][num_tiles * sub_tiles]
     double* stat_partial; // [K][num_tiles]
     double* sq_diff;      // [K][L]
     float* rnorm;         // [K][L]   1/N, or 0 for a zeroed layer
     uint32_t* status;     // [K][L]
+    uint8_t* row_mask;    // [K][total_blocks]  bit j of a block's byte: row j (128 values) holds a nonzero value
+    const uint8_t* row_mask_prev;   // the same for the input behind the previous message, or NULL when unknown
+    int64_t total_blocks; // blocks of 1024 values per worker, all layers
     QodaScalars* scalars;
 };
 
@@ -67,7 +74,8 @@ struct PlanDev {
 int lq_set_error(int code, const char* fmt, ...);
 
 // ---- launchers (each enqueues on `s` and returns the launch status) ----
-cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream_t s);
+// `write_mask`: also record the zero-row masks of `grads` in p.row_mask
+cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write_mask, cudaStream_t s);
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
 // Encode-side tables derived from one level table (rebuilt whenever the levels change).
 struct SearchTables {

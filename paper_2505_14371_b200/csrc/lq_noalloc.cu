@@ -20,7 +20,8 @@ namespace lq {
 namespace {
 
 constexpr int kStaticTiles = 4096;                                    // one fp64 partial per tile
-constexpr int64_t kStaticTileCoords = (int64_t)kTileBlocks * kBlockCoords;
+constexpr int kStaticTileBlocks = 32;                                 // blocks of 1024 values per tile
+constexpr int64_t kStaticTileCoords = (int64_t)kStaticTileBlocks * kBlockCoords;
 constexpr int64_t kStaticMaxCoords = kStaticTiles * kStaticTileCoords;
 constexpr int kMaxDevices = 64;
 
@@ -41,7 +42,7 @@ __device__ __forceinline__ void add_term(double& acc, float v, int q)
     else { double p = a; for (int r = 1; r < q; ++r) p = __dmul_rn(p, a); acc += p; }
 }
 
-// One CTA per tile of kTileBlocks blocks of 1024 values; a lane takes the float4 at 128 j + 4 lane of
+// One CTA per tile of 32 blocks of 1024 values; a lane takes the float4 at 128 j + 4 lane of
 // a block, the same ownership and summation order as the plan-based norm.  A non-finite value
 // makes the partial NaN.
 template <int kMode>
@@ -50,11 +51,11 @@ __global__ void __launch_bounds__(kThreads) static_norm_partial_kernel(const flo
 {
     __shared__ double scratch[kWarps];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t first_block = (int64_t)blockIdx.x * kTileBlocks;
+    const int64_t first_block = (int64_t)blockIdx.x * kStaticTileBlocks;
     const int64_t nblocks = (n + kBlockCoords - 1) / kBlockCoords;
     double acc = 0.0;
     int bad = 0;
-    for (int b = warp; b < kTileBlocks && first_block + b < nblocks; b += kWarps) {
+    for (int b = warp; b < kStaticTileBlocks && first_block + b < nblocks; b += kWarps) {
         const int64_t base = (first_block + b) * kBlockCoords + 4 * lane;
         for (int j = 0; j < 8; ++j) {
             const int64_t pos = base + 128 * j;

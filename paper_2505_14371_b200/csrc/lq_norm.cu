@@ -1,7 +1,9 @@
 // Per-layer L^q norms of K workers' gradients (Section 2.2 of the paper: v is represented by
 // (||v||_q, sign, u)).  Two launches: a streaming pass that leaves one fp64 partial per
 // (worker, tile), and a small pass that adds a layer's partials in a fixed order, so the
-// result does not depend on scheduling.
+// result does not depend on scheduling.  The streaming pass also leaves one byte per block of 1024
+// values whose bit j says whether row j (the 128 values 128 j .. 128 j + 127) holds anything but
+// zeros, so that the encoder, which reads the same values next, can leave all-zero rows unread.
 #include "lq_internal.cuh"
 
 namespace lq {
@@ -28,10 +30,13 @@ __device__ __forceinline__ void accumulate(double& acc, uint32_t& maxbits, float
 }
 
 template <int kMode>
-__global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const float* __restrict__ grads)
+__global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const float* __restrict__ grads,
+                                                                bool write_mask)
 {
     __shared__ double scratch[kThreads / 32];
-    const Tile tile = p.tiles[blockIdx.x];
+    const Tile tile = p.tiles[blockIdx.x / p.sub_tiles];
+    const int sub0 = (blockIdx.x % p.sub_tiles) * kSubBlocks;          // this CTA's blocks of the tile
+    const int sub1 = min(sub0 + kSubBlocks, tile.nblocks);
     const LayerDesc L = p.layers[tile.layer];
     const int k = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -39,9 +44,11 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
 
     double acc = 0.0;
     uint32_t maxbits = 0;
-    for (int b = warp; b < tile.nblocks; b += kWarps) {
+    uint8_t* __restrict__ mask = p.row_mask + (int64_t)k * p.total_blocks + L.block_off;
+    for (int b = sub0 + warp; b < sub1; b += kWarps) {
         const int64_t blk0 = (int64_t)(tile.block0 + b) * kBlockCoords;
         const int64_t base = blk0 + 4 * lane;
+        uint32_t rows = 0;                       // bit j: row j holds a value that is not +-0 (NaN counts)
         if (blk0 + kBlockCoords <= L.size) {
             float4 v[8];
 #pragma unroll
@@ -53,15 +60,24 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
                 accumulate<kMode>(acc, maxbits, v[j].y, p.q);
                 accumulate<kMode>(acc, maxbits, v[j].z, p.q);
                 accumulate<kMode>(acc, maxbits, v[j].w, p.q);
+                const float mag = (fabsf(v[j].x) + fabsf(v[j].y)) + (fabsf(v[j].z) + fabsf(v[j].w));
+                if (__any_sync(0xffffffffu, mag != 0.0f)) rows |= 1u << j;
             }
         } else {
             for (int j = 0; j < 8; ++j) {
                 const int64_t pos = base + 128 * j;
+                float mag = 0.0f;
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (pos + e < L.size) accumulate<kMode>(acc, maxbits, __ldg(g + pos + e), p.q);
+                    if (pos + e < L.size) {
+                        const float x = __ldg(g + pos + e);
+                        accumulate<kMode>(acc, maxbits, x, p.q);
+                        mag += fabsf(x);
+                    }
+                if (__any_sync(0xffffffffu, mag != 0.0f)) rows |= 1u << j;
             }
         }
+        if (write_mask && lane == 0) mask[tile.block0 + b] = (uint8_t)rows;
     }
     if (kMode == 0)   // a non-finite maximum is handed on as NaN so that the final pass sees it
         acc = maxbits >= 0x7f800000u ? __longlong_as_double(0x7ff8000000000000LL)
@@ -75,7 +91,7 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
     } else {
         r = block_reduce<false>(acc, scratch);
     }
-    if (threadIdx.x == 0) p.norm_partial[(int64_t)k * p.num_tiles + blockIdx.x] = r;
+    if (threadIdx.x == 0) p.norm_partial[(int64_t)k * p.num_tiles * p.sub_tiles + blockIdx.x] = r;
 }
 
 // One CTA per (layer, worker): adds the layer's tile partials (thread i takes partials
@@ -86,10 +102,10 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
     __shared__ double scratch[4];
     const int m = blockIdx.x, k = blockIdx.y;
     const LayerDesc L = p.layers[m];
-    const double* part = p.norm_partial + (int64_t)k * p.num_tiles + L.first_tile;
+    const double* part = p.norm_partial + ((int64_t)k * p.num_tiles + L.first_tile) * p.sub_tiles;
     double acc = 0.0;
     int bad = 0;
-    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) {
+    for (int i = threadIdx.x; i < L.ntiles * p.sub_tiles; i += blockDim.x) {
         const double v = part[i];
         if (!(fabs(v) <= 1.7976931348623157e308)) bad = 1;
         if (p.q == 0) acc = fmax(acc, v); else acc += v;
@@ -115,14 +131,14 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
     }
 }
 
-cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, cudaStream_t s)
+cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write_mask, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
-    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
-    if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads);
-    else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads);
-    else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads);
-    else               norm_partial_kernel<3><<<grid, kThreads, 0, s>>>(p, grads);
+    const dim3 grid((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.num_workers);
+    if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
+    else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
+    else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
+    else               norm_partial_kernel<3><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
     return cudaGetLastError();
 }
 

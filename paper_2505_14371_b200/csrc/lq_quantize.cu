@@ -3,7 +3,7 @@
 // with the optional histogram of normalised magnitudes (Algorithm 1 line 4) and the sender-side
 // term of the adaptive step size, sum ||V^_{k,t+1/2} - V^_{k,t-1/2}||^2 (Eq. general_stepsize).
 //
-// Work decomposition: one CTA of 8 warps per (tile, worker); a tile is up to 32 blocks of 1024
+// Work decomposition: one CTA of 8 warps per (tile, worker); a tile is up to 128 blocks of 1024
 // coordinates of one layer, taken round-robin by the warps.  A lane owns the 32 coordinates
 // {128 j + 4 lane + e} of a block (row j = one float4 per lane, 512 contiguous bytes per warp).  Rows
 // travel from global memory into a per-warp ring of 8 rows in shared memory with 16-byte
@@ -20,9 +20,11 @@
 // sit in small tables; every table offset derives from one register (8 * tau, then 4 * symbol with
 // symbol = 2 * idx + sign).
 //
-// A row whose 128 values are all zero (untouched embedding rows) skips the random numbers and the
-// search: its symbols are 0.  If the previous message is all zero there as well, the row adds
-// nothing to the statistic and is skipped entirely.
+// The norm pass, which reads the same values just before, leaves one bit per row of 128 values
+// that says whether the row holds anything but zeros.  An all-zero row (untouched embedding rows)
+// is never fetched, draws no random numbers and needs no search: its symbols are 0.  If the
+// previous message is all zero there as well, the row adds nothing to the statistic and is
+// skipped entirely.
 #include "lq_internal.cuh"
 
 namespace lq {
@@ -40,6 +42,8 @@ struct QuantSmem {
     float tprev[2 * kMaxLevels];     // same for the previous message
     uint32_t hist[LQ_HIST_STRIDE];
     double scratch[kQWarps];
+    uint8_t rows_cur[kTileBlocks];   // per block of the tile: which rows of the input are not all zero
+    uint8_t rows_prev[kTileBlocks];  // the same for the input behind the previous message
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes)
@@ -168,13 +172,16 @@ __device__ __forceinline__ void issue_ragged_block(const WarpCtx& c, int64_t blk
     }
 }
 
-// One block of 1024 coordinates from the ring.  `next` is this lane's first float4 of the block whose
-// rows replace the consumed ones (nullptr: nothing to fetch).  Returns this lane's statistic term.
+// One block of 1024 coordinates from the ring.  `rows` says which of its 8 rows hold anything but
+// zeros (only those were fetched); `next` is this lane's first float4 of the block whose rows
+// replace the consumed ones (nullptr: nothing to fetch) and `next_rows` its row mask; `prev_rows`
+// says which rows may be nonzero in the previous message.  Returns this lane's statistic term.
 template <int B, bool kFast, bool kHist>
 __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const WarpCtx& c,
-                                                 int64_t blk, const float* __restrict__ next,
+                                                 int64_t blk, uint32_t rows, uint32_t prev_rows,
+                                                 const float* __restrict__ next, uint32_t next_rows,
                                                  uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
-                                                 bool prev_live, QuantSmem& sm)
+                                                 QuantSmem& sm)
 {
     constexpr int n = 1 << B, C = B + 1;
     const int lane = c.lane;
@@ -192,14 +199,17 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
 
 #pragma unroll
     for (int j = 0; j < kRingRows; ++j) {
-        cp_async_wait<kRingRows - 1>();
-        float4 v = c.ring_ptr[32 * j];
-        // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
-        v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
-        v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
+        const bool live = (rows >> j) & 1u;              // the same for the whole warp
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (live) {
+            cp_async_wait<kRingRows - 1>();
+            v = c.ring_ptr[32 * j];
+            // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
+            v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
+            v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
+        }
         const float vv[4] = {v.x, v.y, v.z, v.w};
-        const float mag = (fabsf(v.x) + fabsf(v.y)) + (fabsf(v.z) + fabsf(v.w));   // 0 iff all four are 0
-        if (kHist || __any_sync(0xffffffffu, mag != 0.0f)) {
+        if (live) {
             uint32_t x[4];
             philox4x32_10_folded(ctr0 + 32 * j, pc, x);
 #pragma unroll
@@ -246,7 +256,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 const double dd = (double)__fsub_rn(cur, prv);
                 stat = fma(dd, dd, stat);
             }
-        } else if (prev_live) {
+        } else if ((prev_rows >> j) & 1u) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, 4 * j + e));
@@ -254,7 +264,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 stat = fma(dd, dd, stat);
             }
         }
-        if (next) cp_async16(c.ring + 512u * j, next + 128 * j, 16);
+        if (next && ((next_rows >> j) & 1u)) cp_async16(c.ring + 512u * j, next + 128 * j, 16);
         cp_async_commit();
     }
     const int64_t woff = blk * (int64_t)C * 32 + lane;
@@ -288,6 +298,9 @@ __device__ __forceinline__ double zeroed_tile(const Tile& tile, int lane, uint32
     return stat;
 }
 
+// A warp's share of a tile: blocks warp, warp + 8, ...  A block whose rows are all zero in this input and
+// in the input behind the previous message is an all-zero piece of message that adds nothing to the
+// statistic: its words are stored and nothing is read.
 template <int B, bool kFast, bool kHist>
 __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const WarpCtx& c, const Tile& tile,
                                                 uint32_t* __restrict__ out,
@@ -295,37 +308,49 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
 {
     constexpr int C = B + 1;
     const int warp = threadIdx.x >> 5;
-    double stat = 0.0;
-    if (warp >= tile.nblocks) return stat;
-    int64_t blk = tile.block0 + warp;
-    const int64_t end = tile.block0 + tile.nblocks;
     const int64_t nfull = c.size / kBlockCoords;          // blocks below this index lie inside the layer
-    if (blk < nfull) {
-        const float* src = c.g + blk * kBlockCoords + 4 * c.lane;
+    double stat = 0.0;
+    bool primed = false;                                  // the ring holds (or awaits) the rows of block b
+    for (int b = warp; b < tile.nblocks; b += kQWarps) {
+        const int64_t blk = tile.block0 + b;
+        const uint32_t rows = sm.rows_cur[b], prows = sm.rows_prev[b];
+        if ((rows | prows) == 0u) {
+            const int64_t woff = blk * (int64_t)C * 32 + c.lane;
 #pragma unroll
-        for (int j = 0; j < kRingRows; ++j) { cp_async16(c.ring + 512u * j, src + 128 * j, 16); cp_async_commit(); }
-    } else {
-        issue_ragged_block(c, blk);
-    }
-    uint32_t pw[C];
+            for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, 0u);
+            continue;
+        }
+        if (!primed) {
+            if (blk < nfull) {
+                const float* src = c.g + blk * kBlockCoords + 4 * c.lane;
 #pragma unroll
-    for (int w = 0; w < C; ++w) pw[w] = prev ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
-    for (; blk < end; blk += kQWarps) {
-        const int64_t nblk = blk + kQWarps;
-        const bool has_next = nblk < end;
-        uint32_t pn[C];                                   // the next block's previous words, fetched early
+                for (int j = 0; j < kRingRows; ++j) {
+                    if ((rows >> j) & 1u) cp_async16(c.ring + 512u * j, src + 128 * j, 16);
+                    cp_async_commit();
+                }
+            } else {
+                issue_ragged_block(c, blk);
+            }
+        }
+        uint32_t pw[C];
 #pragma unroll
-        for (int w = 0; w < C; ++w)
-            pn[w] = (prev && has_next) ? __ldcs(prev + nblk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
-        uint32_t por = 0u;
+        for (int w = 0; w < C; ++w) pw[w] = (prev && prows) ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
+        // the next block of this warp that has anything in it: its rows replace the consumed ones
+        int nb = b + kQWarps;
+        while (nb < tile.nblocks && (sm.rows_cur[nb] | sm.rows_prev[nb]) == 0u) {
+            const int64_t woff = (tile.block0 + nb) * (int64_t)C * 32 + c.lane;
 #pragma unroll
-        for (int w = 0; w < C; ++w) por |= pw[w];
-        const bool prev_live = __any_sync(0xffffffffu, por != 0u);
+            for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, 0u);
+            nb += kQWarps;
+        }
+        const bool has_next = nb < tile.nblocks;
+        const int64_t nblk = tile.block0 + nb;
+        const uint32_t next_rows = has_next ? sm.rows_cur[nb] : 0u;
         const float* next = (has_next && nblk < nfull) ? c.g + nblk * kBlockCoords + 4 * c.lane : nullptr;
-        stat += quantize_block<B, kFast, kHist>(pc, c, blk, next, out, pw, prev_live, sm);
+        stat += quantize_block<B, kFast, kHist>(pc, c, blk, rows, prows, next, next_rows, out, pw, sm);
+        primed = has_next;
         if (has_next && nblk >= nfull) issue_ragged_block(c, nblk);   // the layer's last, partial block
-#pragma unroll
-        for (int w = 0; w < C; ++w) pw[w] = pn[w];
+        b = nb - kQWarps;                                             // the loop's increment lands on nb
     }
     cp_async_wait<0>();
     return stat;
@@ -365,6 +390,13 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
             sm.lut[i] = st.lut[(int64_t)layer * kLutStride + i];
     if (kHist)
         for (int i = threadIdx.x; i < LQ_HIST_STRIDE; i += blockDim.x) sm.hist[i] = 0;
+    if (threadIdx.x < tile.nblocks) {
+        // with a histogram every coordinate counts, zero or not, so every row is fetched; a previous
+        // message whose masks are unknown is taken as nonzero everywhere
+        const int64_t mb = (int64_t)k * p.total_blocks + L.block_off + tile.block0 + threadIdx.x;
+        sm.rows_cur[threadIdx.x] = kHist ? (uint8_t)0xff : p.row_mask[mb];
+        sm.rows_prev[threadIdx.x] = !prev_packed ? (uint8_t)0 : (p.row_mask_prev ? p.row_mask_prev[mb] : (uint8_t)0xff);
+    }
     __syncthreads();
 
     WarpCtx c;
@@ -381,9 +413,9 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
 
     double stat = 0.0;
     switch (zeroed ? -L.bits : L.bits * 2 + (fast ? 1 : 0)) {
-#define LQ_CASE(BB)                                                                                   \
-    case -BB:        stat = zeroed_tile<BB>(tile, lane, out, prev, sm); break;                        \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(pc, c, tile, out, prev, sm); break; \
+#define LQ_CASE(BB)                                                                              \
+    case -BB:        stat = zeroed_tile<BB>(tile, lane, out, prev, sm); break;                   \
+    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(pc, c, tile, out, prev, sm); break;  \
     case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(pc, c, tile, out, prev, sm); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
