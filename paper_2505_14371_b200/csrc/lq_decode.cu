@@ -11,6 +11,16 @@
 namespace lq {
 
 constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared memory at once
+#ifndef LQ_DEC_PARTS
+#define LQ_DEC_PARTS 2
+#endif
+#ifndef LQ_DEC_CTAS
+#define LQ_DEC_CTAS 4
+#endif
+constexpr int kParts = LQ_DEC_PARTS;            // a block is decoded in kParts pieces of 8 / kParts rows
+constexpr int kPartSyms = 32 / kParts;          // symbols of a lane per piece
+constexpr int kPartRows = 8 / kParts;
+constexpr int kStageBytes = kWarps * 2 * kPartRows * 512;   // per CTA: each warp stages its piece's rows of Y and X_1
 
 
 // Adds up to kWorkerChunk workers' decoded half blocks into acc, in worker order.  Half H of a lane's
@@ -19,13 +29,13 @@ constexpr int kWorkerChunk = 8;   // workers whose value tables sit in shared me
 // that a warp keeps a few KB in flight.  `table[kk]` holds N * l_j at 2j and -N * l_j at 2j + 1 for
 // worker kk of the chunk.
 template <int B, int H>
-__device__ __forceinline__ void decode_accumulate(float (&acc)[16], const uint32_t* __restrict__ words,
+__device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const uint32_t* __restrict__ words,
                                                   int64_t worker_stride, int kc,
                                                   const float (*table)[2 * kMaxLevels])
 {
     constexpr int C = B + 1;
-    constexpr int kFirst = (16 * H * C) >> 5;                         // first and last word of this half
-    constexpr int kLast = ((16 * (H + 1) * C) - 1) >> 5;
+    constexpr int kFirst = (kPartSyms * H * C) >> 5;                  // first and last word of this piece
+    constexpr int kLast = ((kPartSyms * (H + 1) * C) - 1) >> 5;
     uint32_t w[kWorkerChunk][C];
 #pragma unroll
     for (int kk = 0; kk < kWorkerChunk; ++kk)
@@ -37,8 +47,8 @@ __device__ __forceinline__ void decode_accumulate(float (&acc)[16], const uint32
         if (kk < kc) {
             const char* tb = reinterpret_cast<const char*>(table[kk]);
 #pragma unroll
-            for (int p = 0; p < 16; ++p)
-                acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w[kk], 16 * H + p));
+            for (int p = 0; p < kPartSyms; ++p)
+                acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w[kk], kPartSyms * H + p));
         }
     }
 }
@@ -75,14 +85,30 @@ __device__ __forceinline__ void fill_tables(const PlanDev& p, const LayerDesc& L
 template <int B, int H, bool kQoda>
 __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
                                             float (*table)[2 * kMaxLevels], float eta, float invK,
-                                            int64_t blk, bool active, bool& resident)
+                                            int64_t blk, bool active, bool& resident, float4* stage)
 {
     const int lane = threadIdx.x & 31;
     const int K = p.num_workers;
     const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
-    float acc[16];
+    const int64_t base = L.elem_off + blk * kBlockCoords + 4 * lane;
+    const int64_t limit = L.elem_off + L.size;
+    // the state rows of this piece travel to shared memory while the messages are read and decoded
+    // (`stage`: this lane's slots, rows of Y then rows of X_1, 32 float4 apart; only this lane reads them)
+    if (kQoda && active) {
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+        for (int jj = 0; jj < kPartRows; ++jj) {
+            const int64_t pos = base + 128 * (kPartRows * H + jj);
+            if (pos < limit) {
+                cp_async16(dst + 512u * jj, a.Y + pos, 16);
+                cp_async16(dst + 512u * (kPartRows + jj), a.X1 + pos, 16);
+            }
+        }
+        cp_async_commit();
+    }
+    float acc[kPartSyms];
+#pragma unroll
+    for (int i = 0; i < kPartSyms; ++i) acc[i] = 0.0f;
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
         const int kc = min(kWorkerChunk, K - k0);
         if (!resident) fill_tables(p, L, layer, a, table, k0, kc);
@@ -90,12 +116,10 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
         if (active) decode_accumulate<B, H>(acc, a.packed + (int64_t)k0 * p.packed_words + woff, p.packed_words, kc, table);
     }
     if (!active) return;
-
-    const int64_t base = L.elem_off + blk * kBlockCoords + 4 * lane;
-    const int64_t limit = L.elem_off + L.size;
+    if (kQoda) cp_async_wait<0>();
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-        const int64_t pos = base + 128 * (4 * H + jj);
+    for (int jj = 0; jj < kPartRows; ++jj) {
+        const int64_t pos = base + 128 * (kPartRows * H + jj);
         if (pos >= limit) continue;
         float4 g;
         g.x = __fmul_rn(acc[4 * jj + 0], invK);
@@ -104,8 +128,8 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
         g.w = __fmul_rn(acc[4 * jj + 3], invK);
         if (a.gbar) *reinterpret_cast<float4*>(a.gbar + pos) = g;
         if (kQoda) {
-            const float4 y0 = *reinterpret_cast<const float4*>(a.Y + pos);
-            const float4 x1 = __ldg(reinterpret_cast<const float4*>(a.X1 + pos));
+            const float4 y0 = stage[32 * jj];
+            const float4 x1 = stage[32 * (kPartRows + jj)];
             float4 y, x, h;
             y.x = __fsub_rn(y0.x, g.x); y.y = __fsub_rn(y0.y, g.y);
             y.z = __fsub_rn(y0.z, g.z); y.w = __fsub_rn(y0.w, g.w);
@@ -128,22 +152,28 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
     const int warp = threadIdx.x >> 5;
     const float invK = __fdiv_rn(1.0f, (float)p.num_workers);
     bool resident = false;
+    extern __shared__ float4 stage_mem[];                 // [warp][Y rows, X_1 rows][lane]
+    float4* stage = stage_mem + warp * (2 * kPartRows * 32) + (threadIdx.x & 31);
     // each warp takes the tile's blocks round-robin; all warps run the same number of rounds so
     // that the table refills (CTA-wide barriers) stay aligned
     for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
         const bool active = b0 + warp < tile.nblocks;
         const int64_t blk = tile.block0 + b0 + warp;
-        decode_half<B, 0, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident);
-        decode_half<B, 1, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident);
+        decode_half<B, 0, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+        decode_half<B, 1, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+        if (kParts == 4) {
+            decode_half<B, 2 % kParts, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+            decode_half<B, 3 % kParts, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+        }
     }
 }
 
 template <bool kQoda>
-__global__ void __launch_bounds__(kThreads, 4) decode_kernel(PlanDev p, DecodeArgs a)
+__global__ void __launch_bounds__(kThreads, LQ_DEC_CTAS) decode_kernel(PlanDev p, DecodeArgs a)
 {
     __shared__ float table[kWorkerChunk][2 * kMaxLevels];
-    Tile tile = p.tiles[blockIdx.x / p.sub_tiles];                    // this CTA takes one sub-tile of it
-    const int sub0 = (blockIdx.x % p.sub_tiles) * kSubBlocks;
+    Tile tile = p.tiles[blockIdx.x >> p.sub_shift];                    // this CTA takes one sub-tile of it
+    const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
     if (sub0 >= tile.nblocks) return;
     tile.block0 += sub0;
     tile.nblocks = min(kSubBlocks, tile.nblocks - sub0);
@@ -200,8 +230,8 @@ cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float*
 {
     if (p.num_tiles == 0) return cudaSuccess;
     DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
-    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, 0, s>>>(p, a);
-    else      decode_kernel<false><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, 0, s>>>(p, a);
+    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, kStageBytes, s>>>(p, a);
+    else      decode_kernel<false><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, kStageBytes, s>>>(p, a);
     return cudaGetLastError();
 }
 

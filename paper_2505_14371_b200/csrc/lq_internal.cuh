@@ -55,7 +55,8 @@ struct PlanDev {
     int32_t num_tiles;
     int32_t num_workers;
     int32_t q;            // 0 = infinity norm
-    int32_t sub_tiles;    // sub-tiles per tile: the plan's tile size / kSubBlocks
+    int32_t sub_tiles;    // sub-tiles per tile: the plan's tile size / kSubBlocks (1, 2 or 4)
+    int32_t sub_shift;    // log2(sub_tiles)
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;
@@ -133,6 +134,16 @@ __device__ __forceinline__ uint32_t symbol4_at(const uint32_t (&w)[C], int p)
     else             v = __funnelshift_r(w[i], w[i + 1], s - 2);      // s >= 2 whenever a symbol straddles
     return v & mask4;
 }
+
+// 16-byte asynchronous copies global -> shared (completion by commit / wait groups of the issuing thread)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes)
+{
+    // copies `bytes` (0..16) bytes and fills the rest of the 16 with zeros
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ double warp_sum(double v)
 {

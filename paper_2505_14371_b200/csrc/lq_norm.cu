@@ -34,8 +34,8 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
                                                                 bool write_mask)
 {
     __shared__ double scratch[kThreads / 32];
-    const Tile tile = p.tiles[blockIdx.x / p.sub_tiles];
-    const int sub0 = (blockIdx.x % p.sub_tiles) * kSubBlocks;          // this CTA's blocks of the tile
+    const Tile tile = p.tiles[blockIdx.x >> p.sub_shift];
+    const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;          // this CTA's blocks of the tile
     const int sub1 = min(sub0 + kSubBlocks, tile.nblocks);
     const LayerDesc L = p.layers[tile.layer];
     const int k = blockIdx.y;
@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
     for (int b = sub0 + warp; b < sub1; b += kWarps) {
         const int64_t blk0 = (int64_t)(tile.block0 + b) * kBlockCoords;
         const int64_t base = blk0 + 4 * lane;
-        uint32_t rows = 0;                       // bit j: row j holds a value that is not +-0 (NaN counts)
+        uint32_t rows = 0;                       // bit j: this lane's part of row j holds a value that is not +-0 (NaN counts)
         if (blk0 + kBlockCoords <= L.size) {
             float4 v[8];
 #pragma unroll
@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
                 accumulate<kMode>(acc, maxbits, v[j].z, p.q);
                 accumulate<kMode>(acc, maxbits, v[j].w, p.q);
                 const float mag = (fabsf(v[j].x) + fabsf(v[j].y)) + (fabsf(v[j].z) + fabsf(v[j].w));
-                if (__any_sync(0xffffffffu, mag != 0.0f)) rows |= 1u << j;
+                rows |= (mag != 0.0f ? 1u : 0u) << j;
             }
         } else {
             for (int j = 0; j < 8; ++j) {
@@ -74,9 +74,10 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
                         accumulate<kMode>(acc, maxbits, x, p.q);
                         mag += fabsf(x);
                     }
-                if (__any_sync(0xffffffffu, mag != 0.0f)) rows |= 1u << j;
+                rows |= (mag != 0.0f ? 1u : 0u) << j;
             }
         }
+        rows = __reduce_or_sync(0xffffffffu, rows);      // a row is live if any lane's part of it is
         if (write_mask && lane == 0) mask[tile.block0 + b] = (uint8_t)rows;
     }
     if (kMode == 0)   // a non-finite maximum is handed on as NaN so that the final pass sees it

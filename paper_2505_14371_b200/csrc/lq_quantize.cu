@@ -46,15 +46,6 @@ struct QuantSmem {
     uint8_t rows_prev[kTileBlocks];  // the same for the input behind the previous message
 };
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes)
-{
-    // copies `bytes` (0..16) bytes and fills the rest of the 16 with zeros
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
 // x >> K for a constant K.  kMul writes it as the high half of a multiplication, which runs on the
 // multiply-add pipe instead of the integer/logic pipe.
 template <int K, bool kMul>
