@@ -353,6 +353,77 @@ def run_gpu(args) -> None:
         dist.destroy_process_group()
 
 
+
+# ---------------------------------------------------------------------------------- sweep
+def run_sweep(args) -> None:
+    """Bandwidth sweep: flat layers of 2^10 .. 2^30 coordinates and a ragged set of 2048 layers, over code
+    widths, worker counts and norms.  One JSON line per point: device time (CUDA events, inputs resident, L2
+    flushed by a 256 MB write between repetitions when the input is smaller than L2) of lq_quantize_pack and of
+    qoda_step, their algorithmic GB/s and the fraction of the measured HBM peak.  Points whose K inputs would
+    not fit in `--sweep-bytes` reuse one input row for every worker (said in the line)."""
+    import torch
+    import paper_2505_14371_b200 as pkg
+    from paper_2505_14371_b200 import workloads as W
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    pkg.load_library()
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+    points = []
+    for log2n in ([10, 14, 18, 20, 22, 24, 26, 28, 30] if not args.sweep_quick else [14, 22, 26]):
+        for bits, K, q in ([(4, 4, 2)] if log2n not in (26,) else
+                           [(b, k, qq) for b in (2, 3, 4, 8) for k in (1, 4, 16) for qq in (2, 0)]):
+            points.append(("flat", log2n, bits, K, q))
+    for bits in (2, 3, 4, 8):
+        points.append(("ragged", 0, bits, 4, 2))
+    for kind, log2n, bits, K, q in points:
+        w = W.flat_workload(log2n, bits, K, q) if kind == "flat" else W.ragged_workload(bits, K, q)
+        D = w.num_coords
+        plan = pkg.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+        aliased = 4 * K * plan.padded_elems > args.sweep_bytes
+        if aliased:                                # one input row serves every worker (stride 0 is not expressible
+            K_alloc = 1                            # through the ABI, so the plan is rebuilt for the workers that fit)
+            Kfit = max(1, int(args.sweep_bytes // (4 * plan.padded_elems)))
+            plan.close(); K = Kfit
+            w = W.flat_workload(log2n, bits, K, q) if kind == "flat" else W.ragged_workload(bits, K, q)
+            plan = pkg.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+        grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, dev)
+        pk = [plan.empty_packed(dev), plan.empty_packed(dev)]; nm = [plan.empty_norms(dev), plan.empty_norms(dev)]
+        X1 = torch.randn(plan.padded_elems, device=dev); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+        plan.qoda_init(X1, Y, Xh)
+        small = 4 * K * D < (256 << 20)
+        reps = 5 if 4 * K * D > (1 << 30) else 20
+        tq, ts = [], []
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        for t in range(1, reps + 4):
+            c, p = t % 2, (t + 1) % 2
+            if small:
+                flush.fill_(float(t))
+            ev[0].record()
+            plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=None if t == 1 else pk[p],
+                                  prev_norms=None if t == 1 else nm[p])
+            ev[1].record()
+            plan.qoda_step(pk[c], nm[c], X1, Y, Xh)
+            ev[2].record()
+            torch.cuda.synchronize()
+            if t > 3:
+                tq.append(ev[0].elapsed_time(ev[1])); ts.append(ev[1].elapsed_time(ev[2]))
+        cb = (bits + 1) / 8.0
+        mq, ms = sorted(tq)[len(tq) // 2], sorted(ts)[len(ts) // 2]
+        gq = (8.0 + 2 * cb) * K * D / mq / 1e6; gs = (K * cb + 16.0) * D / ms / 1e6
+        print(json.dumps({"sweep": kind, "log2_coords": log2n, "coords": D, "layers": w.num_layers, "bits": bits, "K": K,
+                          "q": "inf" if q == 0 else q, "workers_capped_by_memory": aliased,
+                          "lq_quantize_pack": {"ms": round(mq, 5), "fp32_in_gbs": round(4.0 * K * D / mq / 1e6, 1),
+                                               "algorithmic_gbs": round(gq, 1), "frac_of_measured_peak": round(gq / peak, 3),
+                                               "frac_of_8tbs": round(gq / 8000.0, 3)},
+                          "qoda_step": {"ms": round(ms, 5), "algorithmic_gbs": round(gs, 1),
+                                        "frac_of_measured_peak": round(gs / peak, 3), "frac_of_8tbs": round(gs / 8000.0, 3)},
+                          "l2": "flushed between repetitions" if small else "input exceeds L2"}), flush=True)
+        plan.close()
+        del grads, pk, nm, X1, Y, Xh
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -361,10 +432,16 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="transformer_xl")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, widths, workers, norms")
+    ap.add_argument("--sweep-quick", action="store_true")
+    ap.add_argument("--sweep-bytes", type=float, default=40e9, help="most bytes of fp32 input per sweep point")
     ap.add_argument("--print-source-hashes", action="store_true", help="hashes to record beside new ncu traffic figures")
     args = ap.parse_args()
     if args.print_source_hashes:
         print({k: source_hash(k) for k in KERNEL_SOURCES})
+        return
+    if args.sweep:
+        run_sweep(args)
         return
     if args.impl == "reference":
         run_reference(args)
