@@ -458,3 +458,41 @@ void orc_qoda_update(const float* gbar, const float* X1, float* Y, float* Xhalf,
         Xhalf[i] = fmaf(-eta, gbar[i], x);
     }
 }
+
+/* ------------------------------------------------------------------------------------
+ * Alternative adaptive step sizes (Eq. Alt; appendix "Analysis in Almost Sure Boundedness
+ * Model"):  eta_t = (1 + lambda_{t-2} + mu_{t-2})^(-1/2),  gamma_t = (1 + lambda_{t-2})^(qhat - 1/2),
+ * qhat in (0, 1/4], with the running sums (zero for t <= 0)
+ *   lambda_t = sum_{s<=t} || (1/K) sum_k V^_{k,s+1/2} ||^2      (the appendix's form: the squared
+ *              norm of the aggregate; the main text prints the sum of the workers' squared norms
+ *              over K^2 instead)
+ *   mu_t     = sum_{s<=t} || X_s - X_{s+1} ||^2.
+ * Both norms are taken on fp32 vectors: lambda on the mean gbar the update itself uses, mu on the
+ * fp32 difference of the two iterates; the squares, exact in fp64, are summed in fp64.
+ * ---------------------------------------------------------------------------------- */
+void orc_alt_rates(double lambda, double mu, double qhat, float* eta, float* gamma)
+{
+    *eta = (float)(1.0 / sqrt(1.0 + lambda + mu));
+    *gamma = (float)pow(1.0 + lambda, qhat - 0.5);
+}
+
+double orc_sq_norm(const float* g, int64_t d)
+{
+    double acc = 0.0;
+    for (int64_t i = 0; i < d; ++i) acc += (double)g[i] * (double)g[i];
+    return acc;
+}
+
+/* The optimistic dual averaging update with separate rates (Eq. ODA):
+ *   Y_{t+1} = Y_t - gbar,  X_{t+1} = fma(eta, Y_{t+1}, X_1),  X_{t+3/2} = fma(-gamma, gbar, X_{t+1}). */
+void orc_qoda_update_rates(const float* gbar, const float* X1, float* Y, float* Xhalf, float* X,
+                           float eta, float gamma, int64_t d)
+{
+    for (int64_t i = 0; i < d; ++i) {
+        float y = Y[i] - gbar[i];
+        float x = fmaf(eta, y, X1[i]);
+        Y[i] = y;
+        if (X) X[i] = x;
+        Xhalf[i] = fmaf(-gamma, gbar[i], x);
+    }
+}

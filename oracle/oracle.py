@@ -66,6 +66,10 @@ def lib():
         L.orc_step_size.restype = C.c_double
         L.orc_step_size.argtypes = [C.c_double, C.c_double, C.c_int, f32p]
         L.orc_qoda_update.argtypes = [f32p, f32p, f32p, f32p, f32p, C.c_float, C.c_int64]
+        L.orc_alt_rates.argtypes = [C.c_double, C.c_double, C.c_double, f32p, f32p]
+        L.orc_sq_norm.restype = C.c_double
+        L.orc_sq_norm.argtypes = [f32p, C.c_int64]
+        L.orc_qoda_update_rates.argtypes = [f32p, f32p, f32p, f32p, f32p, C.c_float, C.c_float, C.c_int64]
         _lib = L
     return _lib
 
@@ -191,6 +195,24 @@ def qoda_update(gbar, X1, Y, Xhalf, X, eta) -> None:
                           _p(Xhalf, C.c_float), _p(X, C.c_float), C.c_float(float(eta)), gbar.size)
 
 
+def alt_rates(lam: float, mu: float, qhat: float):
+    """(eta, gamma) of Eq. (Alt) from the running sums lambda and mu."""
+    eta = C.c_float(0); gamma = C.c_float(0)
+    lib().orc_alt_rates(lam, mu, qhat, C.byref(eta), C.byref(gamma))
+    return np.float32(eta.value), np.float32(gamma.value)
+
+
+def sq_norm(g: np.ndarray) -> float:
+    g = _f32(g)
+    return float(lib().orc_sq_norm(_p(g, C.c_float), g.size))
+
+
+def qoda_update_rates(gbar, X1, Y, Xhalf, X, eta, gamma) -> None:
+    """As qoda_update with an extrapolation rate gamma of its own."""
+    lib().orc_qoda_update_rates(_p(gbar, C.c_float), _p(X1, C.c_float), _p(Y, C.c_float), _p(Xhalf, C.c_float),
+                                _p(X, C.c_float), C.c_float(float(eta)), C.c_float(float(gamma)), gbar.size)
+
+
 def uniform_levels(bits: int) -> np.ndarray:
     n = 1 << bits
     return (np.arange(n, dtype=np.float64) / (n - 1)).astype(np.float32)
@@ -216,6 +238,8 @@ class OracleModel:
         self.S = 0.0; self.eta = np.float32(1.0); self.t = 1
         self.prev_decoded = None         # [K][D] decoded V^_{k,t-1/2}
         self.pending_sq = None
+        self.alt_qhat = 0.0              # > 0: the alternative rates of Eq. (Alt) with this exponent
+        self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
 
     # -- ENCODE side (Algorithm 1 line 12) ------------------------------------------------
     def quantize(self, grads: np.ndarray, step: int, want_hist: bool = False):
@@ -269,9 +293,21 @@ class OracleModel:
         self.Xhalf = self.X1.copy(); self.X = self.X1.copy()
         self.S = 0.0; self.eta = np.float32(1.0); self.t = 1
         self.prev_decoded = None
+        self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
 
     def qoda_step(self) -> np.ndarray:
         """Consumes the message of the last quantize() call; returns gbar."""
+        if self.alt_qhat > 0.0:
+            # eta_{t+1}, gamma_{t+1} use the sums through iteration t-1; this iteration's terms come after
+            self.eta, self.gamma = alt_rates(self.lam, self.mu, self.alt_qhat)
+            gbar = aggregate(self.cur_decoded)
+            X_old = self.X.copy()
+            qoda_update_rates(gbar, self.X1, self.Y, self.Xhalf, self.X, self.eta, self.gamma)
+            self.lam += sq_norm(gbar)
+            self.mu += sq_diff(X_old, self.X)
+            self.prev_decoded = self.cur_decoded
+            self.t += 1
+            return gbar
         total = 0.0
         for k in range(self.K):                       # fixed order: worker, then layer
             for m in range(len(self.sizes)):

@@ -205,3 +205,60 @@ def test_qoda_identities_with_quantization(orc):
             gaps[t] = R * np.linalg.norm(_bilinear_operator(A, zbar))
     assert all(0 < b <= a <= 1 for a, b in zip(etas, etas[1:]))
     assert gaps[1500] < 0.5 * gaps[100] < 0.5 * gaps[10]
+
+
+# ---------------------------------------------------------------- alternative step sizes
+def test_alt_rates_closed_form_and_ordering(orc):
+    eta, gamma = orc.alt_rates(3.0, 5.0, 0.25)
+    assert eta == np.float32(1.0 / 3.0) and gamma == np.float32(4.0 ** -0.25)
+    assert orc.alt_rates(0.0, 0.0, 0.1) == (np.float32(1.0), np.float32(1.0))     # eta_1 = eta_2 = gamma_1 = gamma_2 = 1
+    for lam, mu, qh in [(0.5, 0.0, 0.25), (10.0, 3.0, 0.01), (1e6, 1e3, 0.2)]:
+        e, g = orc.alt_rates(lam, mu, qh)
+        assert 0 < e <= g <= 1                                                     # the extrapolation step is the larger one
+    assert orc.sq_norm(np.float32([3.0, -4.0, 2.0 ** -20])) == 25.0 + 2.0 ** -40
+
+
+def test_alt_schedule_hand_worked_two_steps(orc):
+    """One coordinate, K = 1, operator V(x) = x, 8-bit levels so fine that 1 and -1 are levels
+    (no rounding noise): X_1 = 1.  Step 1: X_{3/2} = 1, gbar = 1, eta_2 = gamma_2 = 1, X_2 = 0, X_{5/2} = -1,
+    lambda_1 = 1, mu_1 = 1.  Step 2: gbar = -1, Y_3 = 0, eta_3 = 3^(-1/2), X_3 = 1, gamma_3 = 2^(-1/4),
+    X_{7/2} = 1 + 2^(-1/4); lambda_2 = 2, mu_2 = 2."""
+    model = orc.OracleModel([1], [8], 0, 1, SEED)            # max norm: u = 1 is a level, decoded value exact
+    model.alt_qhat = 0.25
+    model.qoda_init(np.float32([1.0]))
+    for want_g, want_x, want_xh, want_lam, want_mu in [
+            (1.0, 0.0, -1.0, 1.0, 1.0),
+            (-1.0, 1.0, float(np.float32(1.0) + np.float32(2.0 ** -0.25)), 2.0, 2.0)]:
+        V = model.Xhalf.copy()[None, :]
+        model.quantize(V, model.t)
+        g = model.qoda_step()
+        assert float(g[0]) == want_g and float(model.X[0]) == want_x
+        assert abs(float(model.Xhalf[0]) - want_xh) <= 1e-7
+        assert (model.lam, model.mu) == (want_lam, want_mu)
+    assert model.eta == np.float32(3.0 ** -0.5) and model.gamma == np.float32(2.0 ** -0.25)
+
+
+def test_alt_schedule_converges_on_a_noisy_bilinear_game(orc):
+    """Bilinear games are not co-coercive; the alternative rates are the ones the paper proves without
+    that assumption.  The identity X_{t+1} = X_1 - eta_{t+1} sum_s gbar_s holds and the gap of the ergodic
+    average falls."""
+    rng = np.random.default_rng(1)
+    n = 32; D = 2 * n; K = 4
+    A = rng.standard_normal((n, n)) / math.sqrt(n)
+    model = orc.OracleModel([16] * 4, [4] * 4, 2, K, SEED)
+    model.alt_qhat = 0.25
+    X1 = (rng.standard_normal(D) / math.sqrt(D)).astype(np.float32)
+    model.qoda_init(X1)
+    total = np.zeros(D); avg = np.zeros(D); gaps = {}; R = float(np.linalg.norm(X1))
+    for t in range(1, 1501):
+        Xh = model.Xhalf.copy(); avg += Xh
+        V = (_bilinear_operator(A, Xh)[None, :] + 0.1 * rng.standard_normal((K, D))).astype(np.float32)
+        model.quantize(V, t)
+        eta_before = float(model.eta)
+        g = model.qoda_step()
+        total += g.astype(np.float64)
+        assert float(model.eta) <= eta_before and float(model.eta) <= float(model.gamma) <= 1.0
+        assert np.allclose(model.X, X1 - float(model.eta) * total, rtol=0, atol=2e-5)
+        if t in (10, 100, 1500):
+            gaps[t] = R * np.linalg.norm(_bilinear_operator(A, avg / t))
+    assert gaps[1500] < 0.5 * gaps[100] < 0.5 * gaps[10]
