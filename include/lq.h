@@ -140,6 +140,19 @@ int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stre
 int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1,
               float* Y, float* Xhalf, float* X_opt, float* gbar_opt, void* stream);
 
+/* Alternative adaptive step sizes (Eq. Alt with the running sums of the appendix on the almost-sure
+ * boundedness model): with q_hat in (0, 1/4], every following qoda_step uses
+ *   eta_{t+1} = fp32((1 + lambda_{t-1} + mu_{t-1})^(-1/2)),  gamma_{t+1} = fp32((1 + lambda_{t-1})^(q_hat - 1/2)),
+ *   lambda_t = sum_{s<=t} ||gbar_{s+1/2}||^2,  mu_t = sum_{s<=t} ||X_s - X_{s+1}||^2  (fp64 sums of squares of
+ *   fp32 values; both start at 0 in qoda_init, so eta_1 = eta_2 = gamma_1 = gamma_2 = 1),
+ * X_{t+1} = fma(eta_{t+1}, Y_{t+1}, X_1), X_{t+3/2} = fma(-gamma_{t+1}, gbar, X_{t+1}), and adds this
+ * iteration's terms to lambda and mu afterwards.  The statistic of lq_quantize_pack is not used, so
+ * its prev_packed / prev_norms may be NULL.  q_hat = 0 switches back to Eq. (general_stepsize).
+ * Choose the schedule before qoda_init: the two schedules keep separate sums. */
+int qoda_set_alt_rates(lq_plan* plan, double q_hat);
+/* Host copies of lambda, mu and the current gamma; synchronises.  Any output may be NULL. */
+int qoda_get_alt_scalars(const lq_plan* plan, double* lambda, double* mu, double* gamma);
+
 /* Host copies of the QODA scalars (t = index of the next iteration, S, eta); synchronises.
  * Any output may be NULL. */
 int qoda_get_scalars(const lq_plan* plan, int64_t* t, double* S, double* eta);
@@ -181,7 +194,8 @@ int lq_vector_norm_static(const float* v, int64_t n, int32_t q, float* norm_out,
 #define LQ_KERNEL_QODA_SCALARS   4
 #define LQ_KERNEL_DECODE         5
 #define LQ_KERNEL_FIT            6
-#define LQ_NUM_KERNELS           7
+#define LQ_KERNEL_ALT_FINALIZE   7
+#define LQ_NUM_KERNELS           8
 int lq_profile_enable(lq_plan* plan, int32_t enable);
 int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches);
 

@@ -24,11 +24,11 @@ STATUS_NONFINITE = 2
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
+           "qoda_get_scalars", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
-                "decode", "fit"]
+                "decode", "fit", "alt_finalize"]
 
 
 class LqError(RuntimeError):
@@ -62,6 +62,8 @@ def load_library() -> C.CDLL:
     L.qoda_init.argtypes = [vp, vp, vp, vp, vp]
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.qoda_set_alt_rates.argtypes = [vp, C.c_double]
+    L.qoda_get_alt_scalars.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
     L.lq_vector_norm_static.argtypes = [vp, i64, i32, vp, vp, vp]
     L.lq_profile_enable.argtypes = [vp, i32]
@@ -187,6 +189,14 @@ class Plan:
         t, S, eta = C.c_int64(), C.c_double(), C.c_double()
         _check(load_library().qoda_get_scalars(self._h, C.byref(t), C.byref(S), C.byref(eta)))
         return t.value, S.value, eta.value
+
+    def qoda_set_alt_rates(self, q_hat: float) -> None:
+        _check(load_library().qoda_set_alt_rates(self._h, float(q_hat)))
+
+    def qoda_get_alt_scalars(self):
+        lam, mu, gamma = C.c_double(), C.c_double(), C.c_double()
+        _check(load_library().qoda_get_alt_scalars(self._h, C.byref(lam), C.byref(mu), C.byref(gamma)))
+        return lam.value, mu.value, gamma.value
 
     def lq_get_statistics(self):
         """Returns (sq_diff [K][L] float64, status [K][L] int) as torch CPU tensors."""

@@ -68,6 +68,7 @@ struct lq_plan {
     bool have_message = false;
     bool qoda_ready = false;
     bool stat_pending = false;
+    double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
     // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
@@ -86,7 +87,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->dev.alt_partial); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -221,6 +222,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.alt_partial, 2 * (size_t)(ntiles ? ntiles : 1) * (size_t)d.sub_tiles);
     for (int i = 0; i < 2; ++i)
         if (e == cudaSuccess) e = dev_alloc_zero(&p->d_row_mask[i], (size_t)num_workers * (size_t)(blocks ? blocks : 1));
     d.row_mask = p->d_row_mask[0]; d.row_mask_prev = nullptr;
@@ -241,7 +243,8 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
             if (e == cudaSuccess) e = cudaMemcpy(t, host.data(), lev * sizeof(float), cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) {
-        QodaScalars s0{0.0, 0.0, 1, 1.0f, 0.0f};
+        QodaScalars s0{};
+        s0.t = 1; s0.eta = 1.0f; s0.gamma = 1.0f; s0.eta_cur = 1.0f;
         e = cudaMemcpy(d.scalars, &s0, sizeof s0, cudaMemcpyHostToDevice);
     }
     if (e != cudaSuccess) {
@@ -385,7 +388,7 @@ int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float
     lq_plan* mp = const_cast<lq_plan*>(plan);      // the profiler's bookkeeping is not plan state
     LQ_CUDA(timed(mp, LQ_KERNEL_DECODE, s, [&] {
         return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], nullptr, nullptr,
-                             nullptr, nullptr, gbar, false, s);
+                             nullptr, nullptr, gbar, 0, s);
     }));
     return LQ_OK;
 }
@@ -406,12 +409,42 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
     if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
     if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
     cudaStream_t s = (cudaStream_t)stream;
-    LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_qoda_scalars(plan->dev, s); }));
-    LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
-        return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
-                             gbar_opt, true, s);
-    }));
+    if (plan->alt_qhat > 0.0) {
+        const double qh = plan->alt_qhat;
+        LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_alt_scalars(plan->dev, qh, s); }));
+        LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
+            return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
+                                 gbar_opt, 2, s);
+        }));
+        LQ_CUDA(timed(plan, LQ_KERNEL_ALT_FINALIZE, s, [&] { return launch_alt_finalize(plan->dev, s); }));
+    } else {
+        LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_qoda_scalars(plan->dev, s); }));
+        LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
+            return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
+                                 gbar_opt, 1, s);
+        }));
+    }
     plan->stat_pending = false;
+    return LQ_OK;
+}
+
+int qoda_set_alt_rates(lq_plan* plan, double q_hat)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    if (!(q_hat >= 0.0 && q_hat <= 0.25)) return fail(LQ_EINVAL, "q_hat must be in (0, 1/4], or 0 to switch back; got %g", q_hat);
+    plan->alt_qhat = q_hat;
+    return LQ_OK;
+}
+
+int qoda_get_alt_scalars(const lq_plan* plan, double* lambda, double* mu, double* gamma)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    QodaScalars h;
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(&h, plan->dev.scalars, sizeof h, cudaMemcpyDeviceToHost));
+    if (lambda) *lambda = h.lambda;
+    if (mu) *mu = h.mu;
+    if (gamma) *gamma = (double)h.gamma;
     return LQ_OK;
 }
 

@@ -53,6 +53,9 @@ __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const
     }
 }
 
+// The rates one QODA update uses: X_{t+1} = X_1 + eta Y_{t+1}, X_{t+3/2} = X_{t+1} - gamma gbar; eta_cur made X_t.
+struct Rates { float eta, gamma, eta_cur; };
+
 struct DecodeArgs {
     const uint32_t* packed;
     const float* norms;
@@ -82,11 +85,14 @@ __device__ __forceinline__ void fill_tables(const PlanDev& p, const LayerDesc& L
 // One half block: the mean of the K decoded messages for rows 4 H .. 4 H + 3, then the update.
 // Any worker count: the accumulators live across chunks of kWorkerChunk workers; with a single chunk
 // the tables are filled once per CTA (`resident`).
-template <int B, int H, bool kQoda>
+template <int B, int H, int kMode>
 __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
-                                            float (*table)[2 * kMaxLevels], float eta, float invK,
-                                            int64_t blk, bool active, bool& resident, float4* stage)
+                                            float (*table)[2 * kMaxLevels], const Rates& rt, float invK,
+                                            int64_t blk, bool active, bool& resident, float4* stage,
+                                            double& lam_acc, double& mu_acc)
 {
+    constexpr bool kQoda = kMode >= 1, kAlt = kMode == 2;
+    const float eta = rt.eta, gamma = rt.gamma;
     const int lane = threadIdx.x & 31;
     const int K = p.num_workers;
     const int64_t woff = L.word_off + blk * (int64_t)(B + 1) * 32 + lane;
@@ -135,8 +141,23 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
             y.z = __fsub_rn(y0.z, g.z); y.w = __fsub_rn(y0.w, g.w);
             x.x = fmaf(eta, y.x, x1.x); x.y = fmaf(eta, y.y, x1.y);
             x.z = fmaf(eta, y.z, x1.z); x.w = fmaf(eta, y.w, x1.w);
-            h.x = fmaf(-eta, g.x, x.x); h.y = fmaf(-eta, g.y, x.y);
-            h.z = fmaf(-eta, g.z, x.z); h.w = fmaf(-eta, g.w, x.w);
+            h.x = fmaf(-gamma, g.x, x.x); h.y = fmaf(-gamma, g.y, x.y);
+            h.z = fmaf(-gamma, g.z, x.z); h.w = fmaf(-gamma, g.w, x.w);
+            if (kAlt) {
+                // this iteration's terms of lambda = sum ||gbar||^2 and mu = sum ||X_t - X_{t+1}||^2, with
+                // X_t recomputed from Y_t and the rate that produced it; padding coordinates do not count
+                const float gv[4] = {g.x, g.y, g.z, g.w};
+                const float dv[4] = {__fsub_rn(fmaf(rt.eta_cur, y0.x, x1.x), x.x), __fsub_rn(fmaf(rt.eta_cur, y0.y, x1.y), x.y),
+                                     __fsub_rn(fmaf(rt.eta_cur, y0.z, x1.z), x.z), __fsub_rn(fmaf(rt.eta_cur, y0.w, x1.w), x.w)};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (pos + e < limit) {
+                        const double gd = (double)gv[e], dd = (double)dv[e];
+                        lam_acc = fma(gd, gd, lam_acc);
+                        mu_acc = fma(dd, dd, mu_acc);
+                    }
+                }
+            }
             *reinterpret_cast<float4*>(a.Y + pos) = y;
             *reinterpret_cast<float4*>(a.Xhalf + pos) = h;
             if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
@@ -144,10 +165,11 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     }
 }
 
-template <int B, bool kQoda>
+template <int B, int kMode>
 __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
                                                      const Tile& tile, const DecodeArgs& a,
-                                                     float (*table)[2 * kMaxLevels], float eta)
+                                                     float (*table)[2 * kMaxLevels], const Rates& rt,
+                                                     double& lam_acc, double& mu_acc)
 {
     const int warp = threadIdx.x >> 5;
     const float invK = __fdiv_rn(1.0f, (float)p.num_workers);
@@ -159,34 +181,76 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
     for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
         const bool active = b0 + warp < tile.nblocks;
         const int64_t blk = tile.block0 + b0 + warp;
-        decode_half<B, 0, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
-        decode_half<B, 1, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+        decode_half<B, 0, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+        decode_half<B, 1, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
         if (kParts == 4) {
-            decode_half<B, 2 % kParts, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
-            decode_half<B, 3 % kParts, kQoda>(p, L, layer, a, table, eta, invK, blk, active, resident, stage);
+            decode_half<B, 2 % kParts, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+            decode_half<B, 3 % kParts, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
         }
     }
 }
 
-template <bool kQoda>
-__global__ void __launch_bounds__(kThreads, LQ_DEC_CTAS) decode_kernel(PlanDev p, DecodeArgs a)
+template <int kMode>
+__global__ void __launch_bounds__(kThreads, kMode == 2 ? 3 : LQ_DEC_CTAS) decode_kernel(PlanDev p, DecodeArgs a)
 {
     __shared__ float table[kWorkerChunk][2 * kMaxLevels];
+    constexpr bool kAlt = kMode == 2;
+    const int ncta = p.num_tiles * p.sub_tiles;
     Tile tile = p.tiles[blockIdx.x >> p.sub_shift];                    // this CTA takes one sub-tile of it
     const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
-    if (sub0 >= tile.nblocks) return;
+    if (sub0 >= tile.nblocks) {
+        if (kAlt && threadIdx.x == 0) { p.alt_partial[blockIdx.x] = 0.0; p.alt_partial[ncta + blockIdx.x] = 0.0; }
+        return;
+    }
     tile.block0 += sub0;
     tile.nblocks = min(kSubBlocks, tile.nblocks - sub0);
     const int layer = tile.layer;
     const LayerDesc L = p.layers[layer];
-    const float eta = kQoda ? p.scalars->eta : 0.0f;
+    Rates rt{0.0f, 0.0f, 0.0f};
+    if (kMode >= 1) {
+        rt.eta = p.scalars->eta;
+        rt.gamma = kAlt ? p.scalars->gamma : rt.eta;
+        rt.eta_cur = kAlt ? p.scalars->eta_cur : 0.0f;
+    }
+    double lam_acc = 0.0, mu_acc = 0.0;
 
     switch (L.bits) {
-#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kQoda>(p, L, layer, tile, a, table, eta); break;
+#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kMode>(p, L, layer, tile, a, table, rt, lam_acc, mu_acc); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
     }
+    if (kAlt) {                                  // one term per CTA, added in CTA order by the finalize kernel
+        double* scratch = reinterpret_cast<double*>(&table[0][0]);   // the tables are no longer needed (the
+                                                                     // reduction starts with a barrier)
+        const double lam = block_reduce<false>(lam_acc, scratch);
+        const double mu = block_reduce<false>(mu_acc, scratch);
+        if (threadIdx.x == 0) { p.alt_partial[blockIdx.x] = lam; p.alt_partial[ncta + blockIdx.x] = mu; }
+    }
+}
+
+// Eq. (Alt), before the update of iteration t: eta_{t+1} and gamma_{t+1} from the sums through iteration t-1.
+__global__ void alt_scalars_kernel(PlanDev p, double qhat)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        QodaScalars* q = p.scalars;
+        q->eta_cur = q->eta;
+        q->eta = (float)(1.0 / sqrt(1.0 + q->lambda + q->mu));
+        q->gamma = (float)pow(1.0 + q->lambda, qhat - 0.5);
+        q->t = q->t + 1;
+    }
+}
+
+// Eq. (Alt), after the update: adds the CTAs' terms of this iteration to lambda and mu in a fixed order.
+__global__ void __launch_bounds__(256) alt_finalize_kernel(PlanDev p)
+{
+    __shared__ double scratch[8];
+    const int n = p.num_tiles * p.sub_tiles;
+    double lam = 0.0, mu = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) { lam += p.alt_partial[i]; mu += p.alt_partial[n + i]; }
+    const double lam_t = block_reduce<false>(lam, scratch);
+    const double mu_t = block_reduce<false>(mu, scratch);
+    if (threadIdx.x == 0) { p.scalars->lambda += lam_t; p.scalars->mu += mu_t; }
 }
 
 // S_t = S_{t-1} + (sum over workers and layers of the squared differences) / K^2,
@@ -205,6 +269,7 @@ __global__ void __launch_bounds__(256) qoda_scalars_kernel(PlanDev p)
         q->last_delta = delta;
         q->S = q->S + delta;
         q->eta = (float)(1.0 / sqrt(1.0 + q->S));
+        q->gamma = q->eta;
         q->t = q->t + 1;
     }
 }
@@ -221,17 +286,33 @@ __global__ void qoda_init_kernel(PlanDev p, const float* __restrict__ X1, float*
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         QodaScalars* q = p.scalars;
         q->S = 0.0; q->last_delta = 0.0; q->t = 1; q->eta = 1.0f;
+        q->gamma = 1.0f; q->eta_cur = 1.0f; q->lambda = 0.0; q->mu = 0.0;
     }
 }
 
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
-                          float* gbar, bool qoda, cudaStream_t s)
+                          float* gbar, int mode, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
     DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
-    if (qoda) decode_kernel<true><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, kStageBytes, s>>>(p, a);
-    else      decode_kernel<false><<<(unsigned)p.num_tiles * p.sub_tiles, kThreads, kStageBytes, s>>>(p, a);
+    const unsigned grid = (unsigned)p.num_tiles * p.sub_tiles;
+    if (mode == 2)      decode_kernel<2><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    else if (mode == 1) decode_kernel<1><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    else                decode_kernel<0><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s)
+{
+    alt_scalars_kernel<<<1, 32, 0, s>>>(p, qhat);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s)
+{
+    if (p.num_tiles == 0) return cudaSuccess;
+    alt_finalize_kernel<<<1, 256, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -43,7 +43,11 @@ struct QodaScalars {
     double S;             // running sum of Eq. (general_stepsize)
     double last_delta;    // the term added by the last qoda_step
     long long t;          // index of the next iteration
-    float eta;            // eta_t = gamma_t
+    float eta;            // eta_t (= gamma_t under Eq. general_stepsize)
+    float gamma;          // gamma_t (differs from eta_t only under Eq. Alt)
+    double lambda;        // Eq. (Alt): running sum of ||gbar||^2
+    double mu;            // Eq. (Alt): running sum of ||X_s - X_{s+1}||^2
+    float eta_cur;        // Eq. (Alt): the eta that produced the current X_t (needed to recompute X_t from Y_t)
     float pad_;
 };
 
@@ -65,6 +69,7 @@ struct PlanDev {
     double* sq_diff;      // [K][L]
     float* rnorm;         // [K][L]   1/N, or 0 for a zeroed layer
     uint32_t* status;     // [K][L]
+    double* alt_partial;  // [2][num_tiles * sub_tiles]  per-CTA terms of lambda and mu (Eq. Alt)
     uint8_t* row_mask;    // [K][total_blocks]  bit j of a block's byte: row j (128 values) holds a nonzero value
     const uint8_t* row_mask_prev;   // the same for the input behind the previous message, or NULL when unknown
     int64_t total_blocks; // blocks of 1024 values per worker, all layers
@@ -90,9 +95,12 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
                             const float* prev_norms, const float* levels_cur,
                             const float* levels_prev, SearchTables t, cudaStream_t s);
 cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s);
+// mode 0: decode + aggregate only; 1: + QODA update, Eq. (general_stepsize); 2: + QODA update, Eq. (Alt)
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
-                          float* gbar, bool qoda, cudaStream_t s);
+                          float* gbar, int mode, cudaStream_t s);
+cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s);
+cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_qoda_init(const PlanDev& p, const float* X1, float* Y, float* Xhalf,
                              cudaStream_t s);

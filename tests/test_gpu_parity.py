@@ -284,3 +284,40 @@ def test_argument_errors(lqm):
         plan.qoda_step(plan.empty_packed(), plan.empty_norms(), X, X.clone(), X.clone())
     empty = lqm.Plan([], 4, 2, 2, 0)
     assert empty.packed_words == 0
+
+
+def test_qoda_alternative_rates_multi_step(lqm, orc):
+    """Eq. (Alt): eta and gamma from the running sums lambda (||gbar||^2) and mu (||X_s - X_{s+1}||^2), no
+    previous message needed.  30 iterations on ragged layers against the oracle, state compared every step."""
+    sizes = [3000, 100, 2049, 7]
+    plan = lqm.Plan(sizes, [4, 3, 4, 2], 2, 5, SEED)
+    plan.qoda_set_alt_rates(0.25)
+    model = oracle_model(orc, plan)
+    model.alt_qhat = 0.25
+    X1 = _grads(plan, 6)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1); X = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    model.qoda_init(to_unpadded(plan, X1))
+    packed = plan.empty_packed(); norms = plan.empty_norms()
+    for t in range(1, 31):
+        grads = _grads(plan, 2000 + t, 0.3 / math.sqrt(t))
+        plan.lq_quantize_pack(grads, t, packed, norms)
+        plan.qoda_step(packed, norms, X1, Y, Xh, X)
+        ref = model.quantize(to_unpadded(plan, grads), t)
+        assert compare_messages(orc, plan, packed, ref) == (0, 0)
+        model.qoda_step()
+        tt, _, eta = plan.qoda_get_scalars()
+        lam, mu, gamma = plan.qoda_get_alt_scalars()
+        assert tt == t + 1 and eta == float(model.eta) and gamma == float(model.gamma)
+        assert abs(lam - model.lam) <= 1e-12 * model.lam and abs(mu - model.mu) <= 1e-12 * max(model.mu, 1e-300)
+        for got, want in [(Y, model.Y), (Xh, model.Xhalf), (X, model.X)]:
+            assert _close(to_unpadded(plan, got), want, 1e-6)
+    assert 0 < eta < gamma < 1
+    with pytest.raises(lqm.LqError):
+        plan.qoda_set_alt_rates(0.3)
+    # back to the default schedule: a fresh init gives eta = gamma again
+    plan.qoda_set_alt_rates(0.0)
+    plan.qoda_init(X1, Y, Xh)
+    plan.lq_quantize_pack(grads, 1, packed, norms)
+    plan.qoda_step(packed, norms, X1, Y, Xh)
+    _, _, eta = plan.qoda_get_scalars(); _, _, gamma = plan.qoda_get_alt_scalars()
+    assert eta == gamma < 1
