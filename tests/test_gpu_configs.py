@@ -256,3 +256,43 @@ def test_config5_sweep_points(lqm, orc, bits, K, q):
         assert compare_messages(orc, plan, packed, ref) == (0, 0)
         assert np.array_equal(norms.cpu().numpy()[:, :plan.num_layers], ref["norms"])
         assert np.array_equal(to_unpadded(plan, gbar), model.mean_decoded(ref["decoded"]))
+
+
+# --------------------------------------------------------------------------- maximum size
+def test_largest_layer_sampled(lqm, orc):
+    """One layer of 2^31 - 5 coordinates (the plan's limit is 2^31 - 1): byte offsets pass 2^33 and the
+    Philox counter word index/4 passes 2^28.  Sampled blocks - the first, two in the middle, the ragged last -
+    against the oracle; the norm against a library fp64 norm."""
+    if torch.cuda.mem_get_info()[0] < 40e9:
+        pytest.skip("needs about 25 GB of free device memory")
+    d = (1 << 31) - 5
+    plan = lqm.Plan([d], 3, 2, 1, SEED_BIG)
+    assert plan.padded_elems == (1 << 31)
+    grads = torch.empty((1, plan.padded_elems), device="cuda")
+    g = torch.Generator(device="cuda").manual_seed(2031)
+    for s in range(0, plan.padded_elems, 1 << 28):
+        grads[0, s: s + (1 << 28)].normal_(generator=g)
+    grads[0, 5 << 20: 9 << 20] = 0.0                                          # a run of all-zero rows and blocks
+    packed = plan.empty_packed(); norms = plan.empty_norms()
+    gbar = torch.empty(plan.padded_elems, device="cuda")
+    plan.lq_quantize_pack(grads, 9, packed, norms)
+    plan.lq_decode_aggregate(packed, norms, gbar)
+    torch.cuda.synchronize()
+    ref_norm = float(torch.linalg.vector_norm(grads[0, :d].double()))
+    N = float(norms[0, 0])
+    assert abs(N - ref_norm) <= 1e-6 * ref_norm
+    levels = np.array(plan.lq_get_levels(0), np.float32)
+    nblk = (d + 1023) // 1024
+    C = 4
+    for b0 in [0, (6 << 20) // 1024, nblk // 2 + 1, (3 << 29) // 1024 + 7, nblk - 2]:                 # coordinate 3 * 2^29 is byte 6 * 2^30
+        lo = b0 * 1024; hi = min(d, lo + 2048)
+        v = grads[0, lo:hi].cpu().numpy()
+        idx, sg, _ = orc.quantize_layer(v, np.float32(N), levels, SEED_BIG, 9, 0, 0, first_index=lo)
+        words = packed[0, b0 * 32 * C: (b0 + 2) * 32 * C].cpu().numpy().view(np.uint32)
+        gi, gs = orc.unpack_layer(words, hi - lo, 3)
+        assert np.array_equal(gi, idx) and np.array_equal(gs, sg), b0
+        assert np.array_equal(gbar[lo:hi].cpu().numpy(), orc.decode_layer(idx, sg, np.float32(N), levels)), b0
+    assert bool((packed[0, (5 << 20) // 1024 * 32 * C: (9 << 20) // 1024 * 32 * C] == 0).all())
+
+
+SEED_BIG = 0x0123456789ABCDEF
