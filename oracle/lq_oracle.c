@@ -496,3 +496,58 @@ void orc_qoda_update_rates(const float* gbar, const float* X1, float* Y, float* 
         Xhalf[i] = fmaf(-gamma, gbar[i], x);
     }
 }
+
+/* ------------------------------------------------------------------------------------
+ * Code-length accounting (Appendix "Coding Framework").  With F~ the weighted CDF of the
+ * layer's normalised coordinates (taken, as in the fit, piecewise linear from the merged
+ * histogram, plus the point mass at u = 1 of the last bin), the probability that level j is
+ * emitted is  p^_j = int hat_j(u) dF~(u),  hat_j rising linearly from l_{j-1} to l_j and falling
+ * linearly from l_j to l_{j+1} (one-sided at j = 0 and j = n-1): stochastic rounding sends u to
+ * l_tau with probability (l_{tau+1}-u)/(l_{tau+1}-l_tau) and to l_{tau+1} otherwise.
+ * p_out[0..n-1] receives the probabilities (they add up to the total mass, 1).
+ * ---------------------------------------------------------------------------------- */
+int orc_level_probabilities(const uint32_t* hist, int64_t stride, const float* norms, int Z,
+                            int64_t d, const float* level, int n, double* p_out)
+{
+    for (int j = 0; j < n; ++j) p_out[j] = 0.0;
+    if (n < 2 || d <= 0) return 0;
+    double wsum = 0.0;
+    for (int z = 0; z < Z; ++z) wsum += (double)norms[z] * (double)norms[z];
+    if (!(wsum > 0.0)) return 0;
+    for (int i = 0; i < ORC_NUM_BINS; ++i) {
+        double m = 0.0;
+        for (int z = 0; z < Z; ++z)
+            m += (((double)norms[z] * (double)norms[z]) / wsum) * (double)hist[(int64_t)z * stride + i];
+        m /= (double)d;
+        if (m == 0.0) continue;
+        if (i == ORC_NUM_BINS - 1) { p_out[n - 1] += m; continue; }      /* the point mass at u = 1 */
+        double lo = orc_bin_edge(i), hi = orc_bin_edge(i + 1), dens = m / (hi - lo);
+        double x0 = lo;
+        while (x0 < hi) {                  /* cut the bin at the levels inside it */
+            int j = 0;
+            for (int t = 1; t <= n - 2; ++t) if ((double)level[t] <= x0) j = t;
+            double a = level[j], c = level[j + 1];
+            double x1 = c < hi ? c : hi;
+            if (!(x1 > x0)) break;
+            /* on [x0, x1] inside [a, c]: int (c-u)/(c-a) du goes to level j, int (u-a)/(c-a) du to level j+1 */
+            double len = x1 - x0, mid = 0.5 * (x0 + x1);
+            p_out[j]     += dens * len * (c - mid) / (c - a);
+            p_out[j + 1] += dens * len * (mid - a) / (c - a);
+            x0 = x1;
+        }
+    }
+    return 1;
+}
+
+/* Expected message length of one layer in bits as the appendix writes it:
+ *   C_q + (1 - p^_0) d + (H + 1) d,   C_q = 32,   H = - sum_{j=1}^{alpha} p^_j log2 p^_j
+ * (the sum over the interior levels j = 1 .. n-2, as printed).  *nonzeros receives the expected
+ * number of non-zero coordinates (1 - p^_0) d. */
+double orc_expected_code_length(const double* p, int n, int64_t d, double* nonzeros)
+{
+    double H = 0.0;
+    for (int j = 1; j <= n - 2; ++j) if (p[j] > 0.0) H -= p[j] * log2(p[j]);
+    double nz = (1.0 - p[0]) * (double)d;
+    if (nonzeros) *nonzeros = nz;
+    return 32.0 + nz + (H + 1.0) * (double)d;
+}

@@ -66,6 +66,10 @@ def lib():
         L.orc_step_size.restype = C.c_double
         L.orc_step_size.argtypes = [C.c_double, C.c_double, C.c_int, f32p]
         L.orc_qoda_update.argtypes = [f32p, f32p, f32p, f32p, f32p, C.c_float, C.c_int64]
+        L.orc_level_probabilities.restype = C.c_int
+        L.orc_level_probabilities.argtypes = [u32p, C.c_int64, f32p, C.c_int, C.c_int64, f32p, C.c_int, C.POINTER(C.c_double)]
+        L.orc_expected_code_length.restype = C.c_double
+        L.orc_expected_code_length.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_int64, C.POINTER(C.c_double)]
         L.orc_alt_rates.argtypes = [C.c_double, C.c_double, C.c_double, f32p, f32p]
         L.orc_sq_norm.restype = C.c_double
         L.orc_sq_norm.argtypes = [f32p, C.c_int64]
@@ -193,6 +197,22 @@ def qoda_update(gbar, X1, Y, Xhalf, X, eta) -> None:
     """In place on Y, Xhalf (and X when given); all contiguous fp32 arrays of one length."""
     lib().orc_qoda_update(_p(gbar, C.c_float), _p(X1, C.c_float), _p(Y, C.c_float),
                           _p(Xhalf, C.c_float), _p(X, C.c_float), C.c_float(float(eta)), gbar.size)
+
+
+def level_probabilities(hist: np.ndarray, norms, d: int, levels) -> np.ndarray:
+    """Probability of each level being emitted, from the merged histogram (Appendix, coding framework)."""
+    hist = np.ascontiguousarray(hist, np.uint32).reshape(len(norms), -1); norms = _f32(norms); levels = _f32(levels)
+    out = np.zeros(levels.size, np.float64)
+    lib().orc_level_probabilities(_p(hist, C.c_uint32), hist.shape[1], _p(norms, C.c_float), norms.size, d,
+                                  _p(levels, C.c_float), levels.size, _p(out, C.c_double))
+    return out
+
+
+def expected_code_length(p: np.ndarray, d: int):
+    """(expected bits of one layer's message as the appendix writes it, expected non-zero coordinates)."""
+    p = np.ascontiguousarray(p, np.float64); nz = C.c_double(0)
+    bits = lib().orc_expected_code_length(_p(p, C.c_double), p.size, d, C.byref(nz))
+    return float(bits), nz.value
 
 
 def alt_rates(lam: float, mu: float, qhat: float):

@@ -262,3 +262,51 @@ def test_alt_schedule_converges_on_a_noisy_bilinear_game(orc):
         if t in (10, 100, 1500):
             gaps[t] = R * np.linalg.norm(_bilinear_operator(A, avg / t))
     assert gaps[1500] < 0.5 * gaps[100] < 0.5 * gaps[10]
+
+
+# ------------------------------------------------------------------ code-length accounting
+def test_level_probabilities_partition_and_closed_form(orc):
+    rng = np.random.default_rng(21)
+    # any density, any levels: the hat functions add up to one, so the probabilities add up to the mass
+    u = np.abs(rng.standard_normal(40000)) ** 2 * 0.05
+    u = u[u < 1.0]
+    h = _hist_of(orc, u)
+    lv = np.float32([0, 0.01, 0.03, 0.1, 0.2, 0.45, 0.7, 1.0])
+    p = orc.level_probabilities(h[None, :], np.float32([1.0]), u.size, lv)
+    assert abs(p.sum() - 1.0) < 1e-12 and np.all(p >= 0)
+    # uniform density on [2^-4, 1) (whole bins) and levels on bin edges: the integrals are elementary
+    hu = np.zeros(512, np.uint32); d = 0
+    for i in range(1 + 16 * 20, 385):
+        w = int(round((orc.bin_edge(i + 1) - orc.bin_edge(i)) * 2 ** 20)); hu[i] = w; d += w
+    lv = np.float32([0.0, 0.0625, 0.25, 0.5, 1.0])
+    p = orc.level_probabilities(hu[None, :], np.float32([2.0]), d, lv)
+    dens = 1.0 / (1.0 - 0.0625)
+    want = [0.0, dens * (0.25 - 0.0625) / 2, dens * ((0.25 - 0.0625) / 2 + 0.25 / 2), dens * (0.25 / 2 + 0.5 / 2), dens * 0.5 / 2]
+    assert np.allclose(p, want, rtol=0, atol=1e-12)
+    bits, nz = orc.expected_code_length(p, d)
+    H = -sum(x * math.log2(x) for x in want[1:4])
+    assert nz == d and abs(bits - (32 + d + (H + 1) * d)) < 1e-6
+    # the point mass at u = 1 belongs to the last level
+    hp = np.zeros(512, np.uint32); hp[385] = 10
+    assert orc.level_probabilities(hp[None, :], np.float32([1.0]), 10, lv).tolist() == [0, 0, 0, 0, 1.0]
+
+
+def test_emitted_indices_follow_the_level_probabilities(orc):
+    """Quantizing the vector whose histogram was taken: the frequency of each emitted index approaches p^_j
+    (up to the histogram's resolution), and the non-zero count approaches (1 - p^_0) d."""
+    rng = np.random.default_rng(22)
+    d = 200000
+    v = (rng.standard_t(3, d) * 1e-3).astype(np.float32)
+    norm, _ = orc.layer_norm(v, 2)
+    h = orc.histogram_layer(v, norm)
+    lv = orc.fit_levels(h[None, :], np.float32([norm]), d, 16)
+    p = orc.level_probabilities(h[None, :], np.float32([norm]), d, lv)
+    counts = np.zeros(16)
+    R = 20
+    for s in range(R):
+        idx, _, _ = orc.quantize_layer(v, norm, lv, SEED, 500 + s, 0, 0)
+        counts += np.bincount(idx, minlength=16)
+    freq = counts / (R * d)
+    assert np.all(np.abs(freq - p) < 0.01 * p + 2e-4)
+    _, nz = orc.expected_code_length(p, d)
+    assert abs((R * d - counts[0]) / R - nz) < 0.01 * nz
