@@ -140,6 +140,22 @@ int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stre
 int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1,
               float* Y, float* Xhalf, float* X_opt, float* gbar_opt, void* stream);
 
+/* Code-length accounting (appendix on the coding framework).
+ * lq_level_probabilities: for every layer, the probability p^_j that level j is emitted,
+ *   p^_j = int hat_j(u) dF~(u), with F~ the CDF estimate of lq_fit_levels (the num_samples histograms
+ *   merged with the weights N_z^2 / sum N_z^2, linear inside a bin, the last bin a point mass at u = 1) and
+ *   hat_j the rounding probabilities towards l_j from its two neighbouring intervals.  The expected number of
+ *   non-zero coordinates of the layer is (1 - p^_0) d_m and the appendix's expected length in bits is
+ *   32 + (1 - p^_0) d_m + (1 - sum_{j=1}^{n-2} p^_j log2 p^_j) d_m.
+ *   hist dev [num_samples][L][LQ_HIST_STRIDE], norms dev [num_samples][L] as for lq_fit_levels;
+ *   staged = 0: the levels of the latest lq_quantize_pack, 1: the staged levels (latest set / fit);
+ *   probs dev [L][256] doubles out (entries past the layer's level count are 0; a layer without mass gives 0s).
+ * lq_symbol_counts: counts[k][m][j] += number of coordinates of layer m in worker k's message that carry
+ *   level index j (padding excluded).  packed dev [K][W]; counts dev [K][L][256] u32, caller-zeroed. */
+int lq_level_probabilities(const lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
+                           int32_t staged, double* probs, void* stream);
+int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* counts, void* stream);
+
 /* Alternative adaptive step sizes (Eq. Alt with the running sums of the appendix on the almost-sure
  * boundedness model): with q_hat in (0, 1/4], every following qoda_step uses
  *   eta_{t+1} = fp32((1 + lambda_{t-1} + mu_{t-1})^(-1/2)),  gamma_{t+1} = fp32((1 + lambda_{t-1})^(q_hat - 1/2)),

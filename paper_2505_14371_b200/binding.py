@@ -24,7 +24,7 @@ STATUS_NONFINITE = 2
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
+           "qoda_get_scalars", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
@@ -62,6 +62,8 @@ def load_library() -> C.CDLL:
     L.qoda_init.argtypes = [vp, vp, vp, vp, vp]
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.lq_level_probabilities.argtypes = [vp, vp, vp, i32, i32, vp, vp]
+    L.lq_symbol_counts.argtypes = [vp, vp, vp, vp]
     L.qoda_set_alt_rates.argtypes = [vp, C.c_double]
     L.qoda_get_alt_scalars.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
@@ -189,6 +191,14 @@ class Plan:
         t, S, eta = C.c_int64(), C.c_double(), C.c_double()
         _check(load_library().qoda_get_scalars(self._h, C.byref(t), C.byref(S), C.byref(eta)))
         return t.value, S.value, eta.value
+
+    def lq_level_probabilities(self, hist, norms, num_samples: int, probs, staged: bool = False) -> None:
+        _check(load_library().lq_level_probabilities(self._h, _ptr(hist, torch.int32), _ptr(norms, torch.float32),
+                                                     num_samples, 1 if staged else 0, _ptr(probs, torch.float64),
+                                                     _stream()))
+
+    def lq_symbol_counts(self, packed, counts) -> None:
+        _check(load_library().lq_symbol_counts(self._h, _ptr(packed, torch.int32), _ptr(counts, torch.int32), _stream()))
 
     def qoda_set_alt_rates(self, q_hat: float) -> None:
         _check(load_library().qoda_set_alt_rates(self._h, float(q_hat)))

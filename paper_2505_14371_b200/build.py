@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "liblq.so")
 # (source, extra flags).  The level fit is compiled without FMA contraction.
 SOURCES = [("lq_api.cu", []), ("lq_norm.cu", []), ("lq_quantize.cu", []), ("lq_decode.cu", []), ("lq_noalloc.cu", []),
-           ("lq_fit.cu", ["-fmad=false"])]
+           ("lq_fit.cu", ["-fmad=false"]), ("lq_codelen.cu", ["-fmad=false"])]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -428,6 +428,24 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
     return LQ_OK;
 }
 
+int lq_level_probabilities(const lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
+                           int32_t staged, double* probs, void* stream)
+{
+    if (!plan || !hist || !norms || !probs) return fail(LQ_EINVAL, "NULL argument");
+    if (num_samples < 1 || num_samples > LQ_MAX_WORKERS)
+        return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
+    const float* levels = staged ? plan->d_levels_stage : plan->d_levels_enc[plan->cur];
+    LQ_CUDA(launch_level_probabilities(plan->dev, hist, norms, num_samples, levels, probs, (cudaStream_t)stream));
+    return LQ_OK;
+}
+
+int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* counts, void* stream)
+{
+    if (!plan || !packed || !counts) return fail(LQ_EINVAL, "NULL argument");
+    LQ_CUDA(launch_symbol_counts(plan->dev, packed, counts, (cudaStream_t)stream));
+    return LQ_OK;
+}
+
 int qoda_set_alt_rates(lq_plan* plan, double q_hat)
 {
     if (!plan) return fail(LQ_EINVAL, "plan is NULL");

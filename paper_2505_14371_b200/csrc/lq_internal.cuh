@@ -99,6 +99,9 @@ cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
                           float* gbar, int mode, cudaStream_t s);
+cudaError_t launch_level_probabilities(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
+                                       const float* levels, double* probs, cudaStream_t s);
+cudaError_t launch_symbol_counts(const PlanDev& p, const uint32_t* packed, uint32_t* counts, cudaStream_t s);
 cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s);
 cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s);

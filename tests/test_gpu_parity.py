@@ -321,3 +321,43 @@ def test_qoda_alternative_rates_multi_step(lqm, orc):
     plan.qoda_step(packed, norms, X1, Y, Xh)
     _, _, eta = plan.qoda_get_scalars(); _, _, gamma = plan.qoda_get_alt_scalars()
     assert eta == gamma < 1
+
+
+def test_code_length_accounting(lqm, orc):
+    """Level-occurrence probabilities from the histograms and the counts of emitted level indices, against
+    the oracle; and the two against each other: the emitted frequencies follow the probabilities."""
+    from paper_2505_14371_b200 import workloads as W
+    w = W.wgan_workload()
+    sizes = [s // 8 for s in w.layer_sizes] + [0, 5]
+    w.layer_sizes = sizes; w.scales = w.scales + [1.0, 1.0]
+    bits = [3, 4, 2, 8, 3, 4, 5, 3, 1, 4, 4]
+    K = 3
+    plan = lqm.Plan(sizes, bits, 2, K, SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda", workers=K)
+    packed = plan.empty_packed(); norms = plan.empty_norms(); hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels(hist, norms, K)                                        # fitted levels for the second message
+    hist.zero_()
+    plan.lq_quantize_pack(grads, 2, packed, norms, hist=hist)
+    probs = torch.full((plan.num_layers, 256), -1.0, dtype=torch.float64, device="cuda")
+    counts = torch.zeros((K, plan.num_layers, 256), dtype=torch.int32, device="cuda")
+    plan.lq_level_probabilities(hist, norms, K, probs)
+    plan.lq_symbol_counts(packed, counts)
+    torch.cuda.synchronize()
+    model = oracle_model(orc, plan)
+    ref = model.quantize(to_unpadded(plan, grads), 2, want_hist=True)
+    assert compare_messages(orc, plan, packed, ref) == (0, 0)
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    P = probs.cpu().numpy(); Cn = counts.cpu().numpy()
+    for m, (d, b) in enumerate(zip(sizes, bits)):
+        n = 1 << b
+        want = orc.level_probabilities(ref["hist"][:, m, :], ref["norms"][:, m], d, model.levels[m])
+        assert np.allclose(P[m, :n], want, rtol=1e-12, atol=1e-15), m
+        assert np.all(P[m, n:] == 0)
+        for k in range(K):
+            assert np.array_equal(Cn[k, m, :n], np.bincount(ref["idx"][k, off[m]:off[m + 1]], minlength=n)), (k, m)
+        if d > 50000 and b <= 4:
+            # frequencies of one message against the probabilities (weights differ per worker, so loosely)
+            freq = Cn[:, m, :n].sum(axis=0) / (K * d)
+            assert abs(want.sum() - 1.0) < 1e-9
+            assert np.all(np.abs(freq - want) < 0.05 * want + 2e-3), m
