@@ -258,6 +258,7 @@ class OracleModel:
         self.S = 0.0; self.eta = np.float32(1.0); self.t = 1
         self.prev_decoded = None         # [K][D] decoded V^_{k,t-1/2}
         self.pending_sq = None
+        self.norm_scope = "layer"        # "global": one norm over the worker's whole vector (Section 3.1, definition of Q)
         self.alt_qhat = 0.0              # > 0: the alternative rates of Eq. (Alt) with this exponent
         self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
 
@@ -275,10 +276,15 @@ class OracleModel:
         sq = np.zeros((K, Lr), np.float64)
         near = 0
         for k in range(K):
+            if self.norm_scope == "global":      # ||v||_q of the whole vector, shared by every layer of the worker
+                gn, gs = layer_norm(grads[k], self.q)
             for m in range(Lr):
                 a, b = int(self.off[m]), int(self.off[m + 1])
                 v = grads[k, a:b]
-                norms[k, m], status[k, m] = layer_norm(v, self.q)
+                if self.norm_scope == "global":
+                    norms[k, m], status[k, m] = gn, gs
+                else:
+                    norms[k, m], status[k, m] = layer_norm(v, self.q)
                 i_, s_, nr = quantize_layer(v, norms[k, m], self.levels[m], self.seed, step, k, m)
                 near += nr
                 idx[k, a:b], sg[k, a:b] = i_, s_
