@@ -76,6 +76,15 @@ int64_t lq_plan_packed_words(const lq_plan* plan);   /* W, or LQ_EINVAL */
 int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, int64_t* word_off,
                        int32_t* num_levels);
 
+/* Norm scope.  LQ_NORM_PER_LAYER (default): every layer is normalised by its own L^q norm.
+ * LQ_NORM_GLOBAL: the formal definition of Q in Section 3.1 - one norm ||v||_q over the worker's whole vector
+ * (all layers), per-layer level sequences; norms[k][m] then holds that one value for every m, so messages
+ * and every other call keep their format.  A NaN or Inf anywhere then zeroes the worker's whole message.
+ * Takes effect at the next lq_layer_norms / lq_quantize_pack. */
+#define LQ_NORM_PER_LAYER 0
+#define LQ_NORM_GLOBAL    1
+int lq_set_norm_scope(lq_plan* plan, int32_t scope);
+
 /* Level sequence of one layer (Section 3.1: 0 = l_0 < l_1 < ... < l_{n-1} = 1, n = 2^b).
  * host_levels [n] host.  set: validates (n must equal 2^b, increasing by at least 2^-100 per
  * step, ends 0 and 1)

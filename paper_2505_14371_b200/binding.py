@@ -22,7 +22,7 @@ STATUS_ZERO_NORM = 1
 STATUS_NONFINITE = 2
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
-           "lq_plan_layer_info", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
+           "lq_plan_layer_info", "lq_set_norm_scope", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
@@ -53,6 +53,7 @@ def load_library() -> C.CDLL:
     L.lq_plan_padded_elems.argtypes = [vp]; L.lq_plan_padded_elems.restype = i64
     L.lq_plan_packed_words.argtypes = [vp]; L.lq_plan_packed_words.restype = i64
     L.lq_plan_layer_info.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
+    L.lq_set_norm_scope.argtypes = [vp, i32]
     L.lq_set_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_get_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_layer_norms.argtypes = [vp, vp, vp, vp]
@@ -145,6 +146,10 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+    def lq_set_norm_scope(self, scope: str) -> None:
+        """"layer" (default) or "global" (one norm over the worker's whole vector)."""
+        _check(load_library().lq_set_norm_scope(self._h, {"layer": 0, "global": 1}[scope]))
 
     # ---- levels -------------------------------------------------------------------------
     def lq_set_levels(self, layer: int, levels) -> None:

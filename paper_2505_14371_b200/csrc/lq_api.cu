@@ -87,7 +87,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->dev.alt_partial); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -222,6 +222,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_total, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.alt_partial, 2 * (size_t)(ntiles ? ntiles : 1) * (size_t)d.sub_tiles);
     for (int i = 0; i < 2; ++i)
         if (e == cudaSuccess) e = dev_alloc_zero(&p->d_row_mask[i], (size_t)num_workers * (size_t)(blocks ? blocks : 1));
@@ -425,6 +426,14 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
         }));
     }
     plan->stat_pending = false;
+    return LQ_OK;
+}
+
+int lq_set_norm_scope(lq_plan* plan, int32_t scope)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    if (scope != LQ_NORM_PER_LAYER && scope != LQ_NORM_GLOBAL) return fail(LQ_EINVAL, "unknown norm scope %d", scope);
+    plan->dev.global_norm = scope == LQ_NORM_GLOBAL ? 1 : 0;
     return LQ_OK;
 }
 

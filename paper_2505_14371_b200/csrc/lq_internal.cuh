@@ -61,6 +61,7 @@ struct PlanDev {
     int32_t q;            // 0 = infinity norm
     int32_t sub_tiles;    // sub-tiles per tile: the plan's tile size / kSubBlocks (1, 2 or 4)
     int32_t sub_shift;    // log2(sub_tiles)
+    int32_t global_norm;  // 1: one norm per worker over all layers (Section 3.1), 0: one per layer
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;
@@ -69,6 +70,7 @@ struct PlanDev {
     double* sq_diff;      // [K][L]
     float* rnorm;         // [K][L]   1/N, or 0 for a zeroed layer
     uint32_t* status;     // [K][L]
+    double* layer_total;  // [K][L]  per-layer sums (or maxima) before the root, for the global norm
     double* alt_partial;  // [2][num_tiles * sub_tiles]  per-CTA terms of lambda and mu (Eq. Alt)
     uint8_t* row_mask;    // [K][total_blocks]  bit j of a block's byte: row j (128 values) holds a nonzero value
     const uint8_t* row_mask_prev;   // the same for the input behind the previous message, or NULL when unknown

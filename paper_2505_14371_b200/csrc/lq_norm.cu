@@ -114,6 +114,11 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
     bad = __syncthreads_or(bad);
     const double total = p.q == 0 ? block_reduce<true>(acc, scratch) : block_reduce<false>(acc, scratch);
     if (threadIdx.x == 0) {
+        const int64_t o = (int64_t)k * p.num_layers + m;
+        if (p.global_norm) {                     // the layers' totals are combined per worker by norm_global_kernel
+            p.layer_total[o] = bad ? __longlong_as_double(0x7ff8000000000000LL) : total;
+            return;
+        }
         double n64;
         if (p.q == 0 || p.q == 1) n64 = total;
         else if (p.q == 2)        n64 = sqrt(total);
@@ -125,6 +130,49 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
         else if (n < 1.17549435e-38f)
             st = LQ_STATUS_ZERO_NORM;
         if (st) n = 0.0f;
+        norms[o] = n;
+        p.rnorm[o] = st ? 0.0f : __fdiv_rn(1.0f, n);
+        p.status[o] = st;
+    }
+}
+
+// Global norm scope (the formal definition of Q in Section 3.1: one ||v||_q over the whole vector): one CTA per
+// worker combines the layers' totals in layer order and writes the same norm into every layer's slot, so the
+// message keeps its format.  A non-finite value anywhere zeroes the worker's whole message.
+__global__ void __launch_bounds__(128) norm_global_kernel(PlanDev p, float* __restrict__ norms)
+{
+    __shared__ double scratch[4];
+    __shared__ float n_s;
+    __shared__ uint32_t st_s;
+    const int k = blockIdx.x;
+    const double* tot = p.layer_total + (int64_t)k * p.num_layers;
+    double acc = 0.0;
+    int bad = 0;
+    for (int m = threadIdx.x; m < p.num_layers; m += blockDim.x) {
+        const double v = tot[m];
+        if (!(fabs(v) <= 1.7976931348623157e308)) bad = 1;
+        if (p.q == 0) acc = fmax(acc, v); else acc += v;
+    }
+    bad = __syncthreads_or(bad);
+    const double total = p.q == 0 ? block_reduce<true>(acc, scratch) : block_reduce<false>(acc, scratch);
+    if (threadIdx.x == 0) {
+        double n64;
+        if (p.q == 0 || p.q == 1) n64 = total;
+        else if (p.q == 2)        n64 = sqrt(total);
+        else                      n64 = pow(total, 1.0 / (double)p.q);
+        float n = (float)n64;
+        uint32_t st = 0;
+        if (bad || !(fabs(n64) <= 1.7976931348623157e308) || !(fabsf(n) <= 3.402823466e38f))
+            st = LQ_STATUS_NONFINITE;
+        else if (n < 1.17549435e-38f)
+            st = LQ_STATUS_ZERO_NORM;
+        n_s = st ? 0.0f : n;
+        st_s = st;
+    }
+    __syncthreads();
+    const float n = n_s;
+    const uint32_t st = st_s;
+    for (int m = threadIdx.x; m < p.num_layers; m += blockDim.x) {
         const int64_t o = (int64_t)k * p.num_layers + m;
         norms[o] = n;
         p.rnorm[o] = st ? 0.0f : __fdiv_rn(1.0f, n);
@@ -146,6 +194,7 @@ cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s)
 {
     norm_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p, norms);
+    if (p.global_norm) norm_global_kernel<<<(unsigned)p.num_workers, 128, 0, s>>>(p, norms);
     return cudaGetLastError();
 }
 

@@ -361,3 +361,43 @@ def test_code_length_accounting(lqm, orc):
             freq = Cn[:, m, :n].sum(axis=0) / (K * d)
             assert abs(want.sum() - 1.0) < 1e-9
             assert np.all(np.abs(freq - want) < 0.05 * want + 2e-3), m
+
+
+@pytest.mark.parametrize("q", [2, 0, 1])
+def test_global_norm_scope(lqm, orc, q):
+    """One norm over the worker's whole vector (Section 3.1) with per-layer levels: norms, messages, statistic,
+    aggregate and update against the oracle over three steps; a NaN zeroes that worker's whole message."""
+    rng = np.random.default_rng(40 + q)
+    sizes = [5000, 33, 12345, 0, 2048]
+    bits = [4, 3, 2, 4, 3]
+    plan = lqm.Plan(sizes, bits, q, 3, SEED)
+    plan.lq_set_norm_scope("global")
+    for m, b in enumerate(bits):
+        if m % 2 == 0 and b > 1:
+            plan.lq_set_levels(m, _random_levels(rng, 1 << b))
+    model = oracle_model(orc, plan)
+    model.norm_scope = "global"
+    X1 = _grads(plan, 8)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh); model.qoda_init(to_unpadded(plan, X1))
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    scale = torch.tensor(np.repeat([1.0, 0.01, 0.1, 1.0, 3.0], [5024, 64, 12352, 0, 2048]), device="cuda", dtype=torch.float32)
+    for t in range(1, 4):
+        grads = _grads(plan, 300 + t, 0.1) * scale[None, : plan.padded_elems]
+        c, p = t % 2, (t + 1) % 2
+        plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=None if t == 1 else pk[p],
+                              prev_norms=None if t == 1 else nm[p])
+        plan.qoda_step(pk[c], nm[c], X1, Y, Xh)
+        ref = model.quantize(to_unpadded(plan, grads), t)
+        got = nm[c].cpu().numpy()
+        assert np.array_equal(got, ref["norms"]) and np.all(got == got[:, :1])
+        assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+        sq, _ = plan.lq_get_statistics()
+        assert _close(sq.numpy(), ref["sq_diff"], 1e-12)
+        model.qoda_step()
+        assert _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
+    grads[1, plan.elem_offsets[2] + 17] = float("nan")
+    plan.lq_quantize_pack(grads, 9, pk[0], nm[0])
+    torch.cuda.synchronize()
+    _, flags = plan.lq_get_statistics()
+    assert flags[1].tolist() == [lqm.STATUS_NONFINITE] * 5 and int(flags[0].sum()) == 0 and int(flags[2].sum()) == 0
+    assert bool((pk[0][1] == 0).all()) and bool((nm[0][1] == 0).all()) and bool((pk[0][0] != 0).any())
