@@ -15,7 +15,7 @@
  *     the CPU tests (known-answer vectors, closed forms, brute force, invariants).
  *   level fit (orc_fit_levels): the paper states the objective (Section 3.2, the
  *     variance minimisation after Eq. MQV and the CDF weights) but no solver, so the
- *     solver here is this build's own: "parity unpinned" against the paper; it is
+ *     solver here is this implementation's own: "parity unpinned" against the paper; it is
  *     pinned only through properties of the objective (descent, stationarity, the
  *     uniform-density closed form, brute-force search on small cases).
  */
@@ -28,7 +28,7 @@
  * Counter-based random numbers: Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw,
  * "Parallel random numbers: as easy as 1, 2, 3", SC'11).  The paper's quantizer needs one
  * independent uniform per coordinate (Section 3.1, definition of q_l(u)); keying the
- * stream on (seed, step, worker, layer, index) is this build's choice so that a CPU and a
+ * stream on (seed, step, worker, layer, index) is this implementation's choice so that a CPU and a
  * GPU draw the same value for the same coordinate.
  * ---------------------------------------------------------------------------------- */
 void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
@@ -147,7 +147,7 @@ double orc_round_up_probability(double u, const float* level, int n, int* tau_ou
 /* ------------------------------------------------------------------------------------
  * Fixed-width message layout (Section 3.2: a 32-bit float norm, one sign bit and one
  * integer code per coordinate; Section 7.1 footnote: no entropy code on top).
- * The physical layout is this build's:
+ * The physical layout is this implementation's:
  *   every coordinate becomes one symbol of b+1 bits, symbol = 2 * idx + sign (sign in bit 0);
  *   a layer of d coordinates is cut into blocks of 1024 coordinates (the last one
  *   zero-padded); a block is (b+1) planes of 32 words; coordinate c of a block belongs to
@@ -202,7 +202,7 @@ void orc_unpack_layer(const uint32_t* words, int64_t d, int b, uint8_t* idx, uin
 
 /* ------------------------------------------------------------------------------------
  * Histogram of normalised magnitudes of one layer (Algorithm 1, line 4: estimate the
- * distribution of normalised dual vectors).  The binning is this build's: 386 bins,
+ * distribution of normalised dual vectors).  The binning is this implementation's: 386 bins,
  * bin 0 = [0, 2^-24), then 16 bins per octave with edges 2^e * (1 + m/16) up to 1,
  * and the last bin holds u = 1 only.  The bin is found here by comparing against the
  * edges, one by one.
@@ -235,7 +235,7 @@ void orc_histogram_layer(const float* v, int64_t d, float norm, uint32_t* hist)
 /* ------------------------------------------------------------------------------------
  * Level fit (Section 3.2: minimise sum_j int_{l_j}^{l_{j+1}} sigma_Q^2(u; l) dF~(u), with
  * F~ the sum of the Z sampled vectors' CDFs weighted by lambda_z = N_z^2 / sum N_z^2).
- * The paper names no solver; this one is the build's own ("parity unpinned"):
+ * The paper names no solver; this one is this implementation's own ("parity unpinned"):
  *   F~ is taken piecewise linear from the merged histogram (uniform density in a bin);
  *   the mass at u = 1 (last bin) never contributes variance and is left out;
  *   start: quantiles j/(n-1) of the mass above bin 0;
