@@ -288,10 +288,12 @@ static double cdf_inverse(const orc_density* D, double y)
     return D->e[lo] + t * (D->e[lo + 1] - D->e[lo]);
 }
 
+static orc_density D;                 /* single-threaded oracle: static storage is fine */
+static int solve_levels(int n, float* level_out);
+
 int orc_fit_levels(const uint32_t* hist, int64_t stride, const float* norms, int Z,
                    int64_t d, int n, float* level_out)
 {
-    static orc_density D;             /* single-threaded oracle: static storage is fine */
     if (n < 3 || d <= 0) return 0;
     double wsum = 0.0;
     for (int z = 0; z < Z; ++z) wsum += (double)norms[z] * (double)norms[z];
@@ -305,6 +307,35 @@ int orc_fit_levels(const uint32_t* hist, int64_t stride, const float* norms, int
         }
         D.mass[i] = m / (double)d;
     }
+    return solve_levels(n, level_out);
+}
+
+/* One level sequence for a whole type (Section 3.1: coordinates are split into M types, each with
+ * its own sequence; here a type is a set of layers).  The S histograms are those of all (sampled
+ * vector, member layer) pairs of the type, sizes[s] and norms[s] the layer size and norm of each.  The
+ * variance the fit minimises is sum_s N_s^2 sum_{i in s} sigma_Q^2(u_i), so the merged measure weighs
+ * every histogram's counts by N_s^2 (with one member layer this is the CDF weighting of orc_fit_levels);
+ * it is scaled by sum_s N_s^2 d_s to total mass one. */
+int orc_fit_levels_shared(const uint32_t* hist, int64_t stride, const float* norms, const int64_t* sizes,
+                          int S, int n, float* level_out)
+{
+    if (n < 3) return 0;
+    double wd = 0.0;
+    for (int s = 0; s < S; ++s) wd += (double)norms[s] * (double)norms[s] * (double)sizes[s];
+    if (!(wd > 0.0)) return 0;
+    for (int i = 0; i <= 385; ++i) D.e[i] = orc_bin_edge(i);
+    for (int i = 0; i < 385; ++i) {
+        double m = 0.0;
+        for (int s = 0; s < S; ++s)
+            m += ((double)norms[s] * (double)norms[s]) * (double)hist[(int64_t)s * stride + i];
+        D.mass[i] = m / wd;
+    }
+    return solve_levels(n, level_out);
+}
+
+/* The solver proper, on the density left in D. */
+static int solve_levels(int n, float* level_out)
+{
     D.F[0] = 0.0; D.M1[0] = 0.0;
     for (int i = 0; i < 385; ++i) {
         D.F[i + 1] = D.F[i] + D.mass[i];

@@ -57,6 +57,8 @@ def lib():
         L.orc_histogram_layer.argtypes = [f32p, C.c_int64, C.c_float, u32p]
         L.orc_fit_levels.restype = C.c_int
         L.orc_fit_levels.argtypes = [u32p, C.c_int64, f32p, C.c_int, C.c_int64, C.c_int, f32p]
+        L.orc_fit_levels_shared.restype = C.c_int
+        L.orc_fit_levels_shared.argtypes = [u32p, C.c_int64, f32p, C.POINTER(C.c_int64), C.c_int, C.c_int, f32p]
         L.orc_fit_objective.restype = C.c_double
         L.orc_fit_objective.argtypes = [u32p, C.c_int64, f32p, C.c_int, C.c_int64, f32p, C.c_int]
         L.orc_decode_layer.argtypes = [u8p, u8p, C.c_int64, C.c_float, f32p, f32p]
@@ -157,6 +159,16 @@ def fit_levels(hist: np.ndarray, norms, d: int, n: int):
     out = np.zeros(n, np.float32)
     ok = lib().orc_fit_levels(_p(hist, C.c_uint32), hist.shape[1], _p(norms, C.c_float),
                               norms.size, d, n, _p(out, C.c_float))
+    return out if ok else None
+
+
+def fit_levels_shared(hist: np.ndarray, norms, sizes, n: int):
+    """One sequence for a type: hist [S][stride], norms [S], sizes [S] over all (sample, member layer) pairs."""
+    norms = _f32(norms); sizes = np.ascontiguousarray(sizes, np.int64)
+    hist = np.ascontiguousarray(hist, np.uint32).reshape(norms.size, -1)
+    out = np.zeros(n, np.float32)
+    ok = lib().orc_fit_levels_shared(_p(hist, C.c_uint32), hist.shape[1], _p(norms, C.c_float), _p(sizes, C.c_int64),
+                                     norms.size, n, _p(out, C.c_float))
     return out if ok else None
 
 

@@ -310,3 +310,32 @@ def test_emitted_indices_follow_the_level_probabilities(orc):
     assert np.all(np.abs(freq - p) < 0.01 * p + 2e-4)
     _, nz = orc.expected_code_length(p, d)
     assert abs((R * d - counts[0]) / R - nz) < 0.01 * nz
+
+
+# --------------------------------------------------------------- one sequence per type
+def test_shared_fit_reduces_to_the_single_layer_fit_and_minimises_the_summed_variance(orc):
+    rng = np.random.default_rng(41)
+    # one member layer: the same levels as the per-layer fit
+    u = np.abs(rng.standard_normal(30000)) * 0.05
+    h = _hist_of(orc, u[u < 1])
+    a = orc.fit_levels(np.stack([h, h]), np.float32([1.0, 2.0]), u.size, 8)
+    b = orc.fit_levels_shared(np.stack([h, h]), np.float32([1.0, 2.0]), [u.size, u.size], 8)
+    assert np.allclose(a, b, rtol=1e-6, atol=0)
+    # two member layers of different size, norm and shape: the shared sequence minimises
+    # sum_s N_s^2 sum_i sigma_Q^2(u_i) against perturbations and beats either layer's own sequence on that sum
+    u1 = np.abs(rng.standard_normal(20000)) * 0.02
+    u2 = np.abs(rng.laplace(size=5000)) * 0.08; u2 = u2[u2 < 1]
+    h1, h2 = _hist_of(orc, u1), _hist_of(orc, u2)
+    N = np.float32([3.0, 0.5])
+    lv = orc.fit_levels_shared(np.stack([h1, h2]), N, [u1.size, u2.size], 16)
+
+    def total_variance(levels):
+        return float(N[0]) ** 2 * u1.size * _sample_objective(u1, levels) + float(N[1]) ** 2 * u2.size * _sample_objective(u2, levels)
+    best = total_variance(lv)
+    for own in (orc.fit_levels(h1[None], N[:1], u1.size, 16), orc.fit_levels(h2[None], N[1:], u2.size, 16)):
+        assert best <= total_variance(own) * 1.001
+    for _ in range(30):
+        p = lv.astype(np.float64).copy()
+        j = int(rng.integers(1, 15))
+        p[j] += rng.uniform(-0.3, 0.3) * min(p[j] - p[j - 1], p[j + 1] - p[j])
+        assert best <= total_variance(p) * 1.002
