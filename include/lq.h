@@ -127,6 +127,16 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
 int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
                   void* stream);
 
+/* Level update with one sequence per TYPE (Section 3.1: the coordinates are split into M types, each with
+ * its own sequence; a type here is a set of layers).  layer_type host [L]: layers with equal ids form a type and
+ * must have the same code width.  The histograms of all (sample, member layer) pairs of a type are merged with
+ * weights N^2 - the variance being minimised is sum N_s^2 sum_i sigma_Q^2(u_i) - and every member receives the
+ * fitted sequence (staged, like lq_fit_levels; with every layer a type of its own the result is that of
+ * lq_fit_levels up to rounding).  hist, norms, num_samples as for lq_fit_levels.  The id list is copied
+ * before the call returns. */
+int lq_fit_levels_shared(lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
+                         const int32_t* layer_type, void* stream);
+
 /* DECODE + aggregate (Algorithm 1 lines 15 and 17): gbar = (1/K) sum_k N_k * sign * l_idx,
  * summed in fp32 in worker order, with the levels of the latest lq_quantize_pack.
  *   packed dev [K][W];  norms dev [K][L];  gbar dev [D_pad] out. */

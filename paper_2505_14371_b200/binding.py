@@ -23,7 +23,7 @@ STATUS_NONFINITE = 2
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_norm_scope", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
-           "lq_quantize_pack", "lq_fit_levels", "lq_decode_aggregate", "qoda_init", "qoda_step",
+           "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
@@ -59,6 +59,7 @@ def load_library() -> C.CDLL:
     L.lq_layer_norms.argtypes = [vp, vp, vp, vp]
     L.lq_quantize_pack.argtypes = [vp, vp, u32, vp, vp, vp, vp, vp, vp]
     L.lq_fit_levels.argtypes = [vp, vp, vp, i32, vp]
+    L.lq_fit_levels_shared.argtypes = [vp, vp, vp, i32, C.POINTER(i32), vp]
     L.lq_decode_aggregate.argtypes = [vp, vp, vp, vp, vp]
     L.qoda_init.argtypes = [vp, vp, vp, vp, vp]
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -177,6 +178,11 @@ class Plan:
     def lq_fit_levels(self, hist, norms, num_samples: int) -> None:
         _check(load_library().lq_fit_levels(self._h, _ptr(hist, torch.int32), _ptr(norms, torch.float32),
                                             num_samples, _stream()))
+
+    def lq_fit_levels_shared(self, hist, norms, num_samples: int, layer_type: Sequence[int]) -> None:
+        ids = (C.c_int32 * max(self.num_layers, 1))(*[int(t) for t in layer_type])
+        _check(load_library().lq_fit_levels_shared(self._h, _ptr(hist, torch.int32), _ptr(norms, torch.float32),
+                                                   num_samples, ids, _stream()))
 
     def lq_decode_aggregate(self, packed, norms, gbar) -> None:
         _check(load_library().lq_decode_aggregate(self._h, _ptr(packed, torch.int32), _ptr(norms, torch.float32),

@@ -68,6 +68,9 @@ struct lq_plan {
     bool have_message = false;
     bool qoda_ready = false;
     bool stat_pending = false;
+    int32_t* d_member_off = nullptr;       // [L + 1] and [L]: the member lists of lq_fit_levels_shared
+    int32_t* d_member_layer = nullptr;
+    std::vector<int32_t> h_members;        // host staging of both lists (kept alive for the asynchronous copy)
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
@@ -87,7 +90,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -223,6 +226,8 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_total, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_member_off, nl + 1);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_member_layer, nl);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.alt_partial, 2 * (size_t)(ntiles ? ntiles : 1) * (size_t)d.sub_tiles);
     for (int i = 0; i < 2; ++i)
         if (e == cudaSuccess) e = dev_alloc_zero(&p->d_row_mask[i], (size_t)num_workers * (size_t)(blocks ? blocks : 1));
@@ -377,6 +382,52 @@ int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32
     cudaStream_t s = (cudaStream_t)stream;
     LQ_CUDA(timed(plan, LQ_KERNEL_FIT, s, [&] {
         return launch_fit(plan->dev, hist, norms, num_samples, plan->d_levels_stage, s);
+    }));
+    plan->stage_dirty = true;
+    return LQ_OK;
+}
+
+int lq_fit_levels_shared(lq_plan* plan, const uint32_t* hist, const float* norms, int32_t num_samples,
+                         const int32_t* layer_type, void* stream)
+{
+    if (!plan || !hist || !norms || !layer_type) return fail(LQ_EINVAL, "NULL argument");
+    if (num_samples < 1 || num_samples > LQ_MAX_WORKERS)
+        return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
+    const int L = plan->dev.num_layers;
+    if (L == 0) return LQ_OK;
+    // member lists: layers grouped by type id, types in order of first appearance
+    std::vector<int32_t> ids, off(1, 0), members;
+    try {
+        for (int m = 0; m < L; ++m) {
+            bool seen = false;
+            for (int32_t id : ids) if (id == layer_type[m]) { seen = true; break; }
+            if (!seen) ids.push_back(layer_type[m]);
+        }
+        for (int32_t id : ids) {
+            int first = -1;
+            for (int m = 0; m < L; ++m) {
+                if (layer_type[m] != id) continue;
+                if (first < 0) first = m;
+                else if (plan->layers[(size_t)m].nlevels != plan->layers[(size_t)first].nlevels)
+                    return fail(LQ_EINVAL, "layers %d and %d share type %d but not their code width", first, m, id);
+                members.push_back(m);
+            }
+            off.push_back((int32_t)members.size());
+        }
+        plan->h_members = off;
+        plan->h_members.insert(plan->h_members.end(), members.begin(), members.end());
+    } catch (const std::bad_alloc&) {
+        return fail(LQ_ENOMEM, "host allocation failed");
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    const int num_types = (int)ids.size();
+    LQ_CUDA(cudaMemcpyAsync(plan->d_member_off, plan->h_members.data(), off.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, s));
+    LQ_CUDA(cudaMemcpyAsync(plan->d_member_layer, plan->h_members.data() + off.size(), members.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, s));
+    LQ_CUDA(timed(plan, LQ_KERNEL_FIT, s, [&] {
+        return launch_fit_shared(plan->dev, hist, norms, num_samples, plan->d_levels_stage, plan->d_member_off,
+                                 plan->d_member_layer, num_types, s);
     }));
     plan->stage_dirty = true;
     return LQ_OK;

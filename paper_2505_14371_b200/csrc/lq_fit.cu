@@ -69,16 +69,55 @@ __device__ double cdf_inv(const FitSmem& s, double y)
     return s.e[lo] + t * (s.e[lo + 1] - s.e[lo]);
 }
 
+// Per-layer mode (member_off == nullptr): CTA m fits layer m.  Shared mode: CTA t fits one sequence for type t,
+// whose member layers are member_layer[member_off[t] .. member_off[t+1]) (all with the same level count): the
+// histograms of all (sample, member) pairs are merged with weights N^2 (the variance to minimise is
+// sum N_s^2 sum_i sigma^2(u_i)), scaled by sum N_s^2 d_s, and the result goes to every member.
 __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, const uint32_t* __restrict__ hist,
                                                                  const float* __restrict__ norms, int Z,
-                                                                 float* __restrict__ levels_stage)
+                                                                 float* __restrict__ levels_stage,
+                                                                 const int32_t* __restrict__ member_off,
+                                                                 const int32_t* __restrict__ member_layer)
 {
     __shared__ FitSmem s;
-    const int m = blockIdx.x;
+    const bool shared_fit = member_off != nullptr;
+    const int m0 = shared_fit ? member_off[blockIdx.x] : 0, m1 = shared_fit ? member_off[blockIdx.x + 1] : 0;
+    if (shared_fit && m1 <= m0) return;
+    const int m = shared_fit ? member_layer[m0] : blockIdx.x;
     const LayerDesc L = p.layers[m];
     const int n = L.nlevels;
-    if (n < 3 || L.size <= 0) return;
+    if (n < 3) return;
     const int tid = threadIdx.x;
+
+    if (shared_fit) {
+        if (tid == 0) {
+            double wd = 0.0;
+            for (int z = 0; z < Z; ++z)
+                for (int j = m0; j < m1; ++j) {
+                    const int mm = member_layer[j];
+                    const double w = (double)norms[(int64_t)z * p.num_layers + mm];
+                    wd += w * w * (double)p.layers[mm].size;
+                }
+            s.moved = wd;
+            s.ok = wd > 0.0;
+        }
+        __syncthreads();
+        if (!s.ok) return;
+        const double wd = s.moved;
+        for (int i = tid; i <= kBins; i += kFitThreads) s.e[i] = bin_edge(i);
+        for (int i = tid; i < kBins; i += kFitThreads) {
+            double acc = 0.0;
+            for (int z = 0; z < Z; ++z)
+                for (int j = m0; j < m1; ++j) {
+                    const int mm = member_layer[j];
+                    const double w = (double)norms[(int64_t)z * p.num_layers + mm];
+                    acc += (w * w) * (double)hist[((int64_t)z * p.num_layers + mm) * LQ_HIST_STRIDE + i];
+                }
+            s.mass[i] = acc / wd;
+        }
+        __syncthreads();
+    } else {
+    if (L.size <= 0) return;
 
     if (tid == 0) {
         double wsum = 0.0;
@@ -104,6 +143,7 @@ __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, cons
         s.mass[i] = acc / (double)L.size;
     }
     __syncthreads();
+    }
     if (tid == 0) {
         s.F[0] = 0.0; s.M1[0] = 0.0;
         for (int i = 0; i < kBins; ++i) {
@@ -174,6 +214,10 @@ __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, cons
             const float ce = nextafterf(out[j + 1], -1.0f);
             if (out[j] > ce) out[j] = ce;
         }
+        for (int jm = m0 + 1; jm < m1; ++jm) {             // the other members of the type receive the same sequence
+            float* dst = levels_stage + (int64_t)member_layer[jm] * kLevelStride;
+            for (int j = 0; j < n; ++j) dst[j] = out[j];
+        }
     }
 }
 
@@ -181,7 +225,18 @@ cudaError_t launch_fit(const PlanDev& p, const uint32_t* hist, const float* norm
                        float* levels_stage, cudaStream_t s)
 {
     if (p.num_layers == 0) return cudaSuccess;
-    fit_levels_kernel<<<(unsigned)p.num_layers, kFitThreads, 0, s>>>(p, hist, norms, num_samples, levels_stage);
+    fit_levels_kernel<<<(unsigned)p.num_layers, kFitThreads, 0, s>>>(p, hist, norms, num_samples, levels_stage,
+                                                                     nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fit_shared(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
+                              float* levels_stage, const int32_t* member_off, const int32_t* member_layer,
+                              int num_types, cudaStream_t s)
+{
+    if (num_types == 0) return cudaSuccess;
+    fit_levels_kernel<<<(unsigned)num_types, kFitThreads, 0, s>>>(p, hist, norms, num_samples, levels_stage,
+                                                                  member_off, member_layer);
     return cudaGetLastError();
 }
 

@@ -111,6 +111,9 @@ cudaError_t launch_qoda_init(const PlanDev& p, const float* X1, float* Y, float*
                              cudaStream_t s);
 cudaError_t launch_fit(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
                        float* levels_stage, cudaStream_t s);
+cudaError_t launch_fit_shared(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
+                              float* levels_stage, const int32_t* member_off, const int32_t* member_layer,
+                              int num_types, cudaStream_t s);
 
 // ---- device helpers ----
 #ifdef __CUDACC__

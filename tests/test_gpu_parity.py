@@ -401,3 +401,39 @@ def test_global_norm_scope(lqm, orc, q):
     _, flags = plan.lq_get_statistics()
     assert flags[1].tolist() == [lqm.STATUS_NONFINITE] * 5 and int(flags[0].sum()) == 0 and int(flags[2].sum()) == 0
     assert bool((pk[0][1] == 0).all()) and bool((nm[0][1] == 0).all()) and bool((pk[0][0] != 0).any())
+
+
+def test_fit_levels_shared_by_type(lqm, orc):
+    """One sequence per type: layers 0, 2, 5 (4 bits) form one type, 1 and 3 (3 bits) another, 4 is alone.
+    Levels against the oracle's shared fit, every member receives the same sequence, and a type whose members
+    disagree on the code width is refused."""
+    from paper_2505_14371_b200 import workloads as W
+    sizes = [30000, 7000, 12345, 4096, 9000, 100]
+    bits = [4, 3, 4, 3, 5, 4]
+    types = [7, 2, 7, 2, 9, 7]
+    K = 4
+    w = W.Workload("typed", sizes, bits=4, q=2, num_workers=K, dist="student3",
+                   scales=[1e-2, 1e-3, 3e-2, 1e-4, 1e-1, 1e-3], config_id=6)
+    plan = lqm.Plan(sizes, bits, 2, K, SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda")
+    packed = plan.empty_packed(); norms = plan.empty_norms(); hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels_shared(hist, norms, K, types)
+    h = hist.cpu().numpy().view(np.uint32); n = norms.cpu().numpy()
+    got = [np.array(plan.lq_get_levels(m), np.float32) for m in range(len(sizes))]
+    for tid in sorted(set(types)):
+        members = [m for m, t in enumerate(types) if t == tid]
+        hs = np.stack([h[z, m] for z in range(K) for m in members])
+        ns = np.float32([n[z, m] for z in range(K) for m in members])
+        ds = [sizes[m] for z in range(K) for m in members]
+        want = orc.fit_levels_shared(hs, ns, ds, 1 << bits[members[0]])
+        for m in members:
+            assert np.allclose(got[m], want, rtol=1e-6, atol=0), (tid, m)
+            assert np.array_equal(got[m], got[members[0]])
+    # the shared sequences are what the next message is encoded with
+    model = oracle_model(orc, plan)
+    plan.lq_quantize_pack(grads, 2, packed, norms)
+    ref = model.quantize(to_unpadded(plan, grads), 2)
+    assert compare_messages(orc, plan, packed, ref) == (0, 0)
+    with pytest.raises(lqm.LqError):
+        plan.lq_fit_levels_shared(hist, norms, K, [1, 1, 1, 1, 1, 1])
