@@ -203,7 +203,8 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     PlanDev& d = p->dev;
     d.num_layers = num_layers; d.num_tiles = (int32_t)ntiles; d.num_workers = num_workers; d.q = q;
     d.sub_tiles = tile_blocks / kSubBlocks;
-    d.sub_shift = d.sub_tiles == 4 ? 2 : (d.sub_tiles == 2 ? 1 : 0);
+    d.sub_shift = 0;
+    while ((1 << d.sub_shift) < d.sub_tiles) ++d.sub_shift;
     d.padded_elems = elem; d.packed_words = word; d.total_blocks = blocks;
     d.seed_lo = (uint32_t)seed; d.seed_hi = (uint32_t)(seed >> 32);
 
