@@ -12,6 +12,8 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that
  *    take a stream only enqueue work on it and return; they do not synchronise unless
  *    stated.  Calls on one plan must be issued in stream order by the caller.
+ *  - fp32 rows (grads, X1, Y, Xhalf, X, gbar) must start on a 16-byte boundary, message and norm
+ *    buffers on a 4-byte boundary; a misaligned pointer is refused with LQ_EINVAL.
  *  - Argument errors are reported synchronously.  Data problems (NaN/Inf input, zero
  *    norm) never fault: they set per-(worker, layer) status flags, see lq_get_statistics.
  *
@@ -109,9 +111,14 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
  *     lq_quantize_pack call (dev [K][W], [K][L]), or both NULL when there is none
  *     (V^_{k,1/2} = 0).  Used for the step-size statistic
  *     sum_k ||V^_{k,t+1/2} - V^_{k,t-1/2}||^2 of Eq. (general_stepsize), which is left
- *     inside the plan for the next qoda_step.  The previous message is decoded with the
- *     levels it was encoded with, even if the levels were changed in between.
- *   prev_packed must not alias packed. */
+ *     inside the plan for the next qoda_step: per coordinate the fp32 difference of the two
+ *     decoded fp32 values, its square summed in fp64.  The previous message is decoded with the
+ *     levels it was encoded with, even if the levels were changed in between.  It MUST be the
+ *     output of this plan's previous lq_quantize_pack call: the plan remembers which rows of
+ *     that call's input were all zero and does not read the corresponding words again.
+ *   prev_packed must not alias packed.
+ *   The sign of a coordinate is (v < 0): +0 and -0 both give symbol 0, so rows of zeros (of either
+ *   sign) become all-zero words; such rows are detected by the norm pass and not read again. */
 int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t* packed,
                      float* norms, uint32_t* hist, const uint32_t* prev_packed,
                      const float* prev_norms, void* stream);

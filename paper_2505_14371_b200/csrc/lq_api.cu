@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdint>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -38,6 +39,14 @@ int lq::lq_set_error(int code, const char* fmt, ...)
 }
 
 namespace {
+
+// Vector loads, stores and asynchronous copies need 16-byte aligned rows (D_pad is a multiple of 32 elements,
+// so an aligned base keeps every row and layer aligned); message words and norms are read as 32-bit values.
+bool misaligned(const void* p, size_t a) { return p && (reinterpret_cast<uintptr_t>(p) % a) != 0; }
+#define LQ_ALIGNED(ptr, a)                                                                   \
+    do {                                                                                      \
+        if (misaligned(ptr, a)) return fail(LQ_EINVAL, #ptr " must be %d-byte aligned", (int)(a)); \
+    } while (0)
 
 #define LQ_CUDA(expr)                                                                         \
     do {                                                                                      \
@@ -327,6 +336,7 @@ int lq_get_levels(const lq_plan* plan, int32_t layer, float* host_levels, int32_
 int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream)
 {
     if (!plan || !grads || !norms) return fail(LQ_EINVAL, "NULL argument");
+    LQ_ALIGNED(grads, 16); LQ_ALIGNED(norms, 4);
     if (plan->dev.num_layers == 0) return LQ_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const PlanDev& d = plan->dev;
@@ -342,6 +352,8 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     if ((prev_packed == nullptr) != (prev_norms == nullptr))
         return fail(LQ_EINVAL, "prev_packed and prev_norms must both be given or both be NULL");
     if (prev_packed == packed) return fail(LQ_EINVAL, "prev_packed must not alias packed");
+    LQ_ALIGNED(grads, 16); LQ_ALIGNED(packed, 4); LQ_ALIGNED(norms, 4); LQ_ALIGNED(hist, 4);
+    LQ_ALIGNED(prev_packed, 4); LQ_ALIGNED(prev_norms, 4);
     if (plan->dev.num_layers == 0) return LQ_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const size_t lev_bytes = (size_t)plan->dev.num_layers * kLevelStride * sizeof(float);
@@ -437,6 +449,7 @@ int lq_fit_levels_shared(lq_plan* plan, const uint32_t* hist, const float* norms
 int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float* norms, float* gbar, void* stream)
 {
     if (!plan || !packed || !norms || !gbar) return fail(LQ_EINVAL, "NULL argument");
+    LQ_ALIGNED(packed, 4); LQ_ALIGNED(norms, 4); LQ_ALIGNED(gbar, 16);
     cudaStream_t s = (cudaStream_t)stream;
     lq_plan* mp = const_cast<lq_plan*>(plan);      // the profiler's bookkeeping is not plan state
     LQ_CUDA(timed(mp, LQ_KERNEL_DECODE, s, [&] {
@@ -449,6 +462,7 @@ int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float
 int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stream)
 {
     if (!plan || !X1 || !Y || !Xhalf) return fail(LQ_EINVAL, "NULL argument");
+    LQ_ALIGNED(X1, 16); LQ_ALIGNED(Y, 16); LQ_ALIGNED(Xhalf, 16);
     LQ_CUDA(launch_qoda_init(plan->dev, X1, Y, Xhalf, (cudaStream_t)stream));
     plan->qoda_ready = true;
     plan->stat_pending = false;
@@ -459,6 +473,8 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
               float* Xhalf, float* X_opt, float* gbar_opt, void* stream)
 {
     if (!plan || !packed || !norms || !X1 || !Y || !Xhalf) return fail(LQ_EINVAL, "NULL argument");
+    LQ_ALIGNED(packed, 4); LQ_ALIGNED(norms, 4); LQ_ALIGNED(X1, 16); LQ_ALIGNED(Y, 16); LQ_ALIGNED(Xhalf, 16);
+    LQ_ALIGNED(X_opt, 16); LQ_ALIGNED(gbar_opt, 16);
     if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
     if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
     cudaStream_t s = (cudaStream_t)stream;

@@ -284,6 +284,13 @@ def test_argument_errors(lqm):
         plan.qoda_step(plan.empty_packed(), plan.empty_norms(), X, X.clone(), X.clone())
     empty = lqm.Plan([], 4, 2, 2, 0)
     assert empty.packed_words == 0
+    # misaligned rows are refused before any kernel could fault on them
+    big = torch.zeros(2 * plan.padded_elems + 8, device="cuda")
+    packed, norms = plan.empty_packed(), plan.empty_norms()
+    with pytest.raises(lqm.LqError, match="aligned"):
+        plan.lq_quantize_pack(big[1: 1 + plan.padded_elems].view(1, -1), 1, packed, norms)
+    with pytest.raises(lqm.LqError, match="aligned"):
+        plan.qoda_init(big[: plan.padded_elems], big[plan.padded_elems + 1: 2 * plan.padded_elems + 1], X.clone())
 
 
 def test_qoda_alternative_rates_multi_step(lqm, orc):
