@@ -582,3 +582,117 @@ double orc_expected_code_length(const double* p, int n, int64_t d, double* nonze
     if (nonzeros) *nonzeros = nz;
     return 32.0 + nz + (H + 1.0) * (double)d;
 }
+
+/* ------------------------------------------------------------------------------------
+ * Lossless prefix code on the level symbols (appendix, "Further Details on Coding Framework":
+ * with the symbol frequencies known or estimated, classical Huffman coding).
+ *
+ * orc_huffman_lengths: code lengths of a Huffman code for n <= 256 symbols with weights w
+ * (probabilities or counts).  Every symbol receives a code word, also those of weight zero (an
+ * estimated distribution may miss a symbol that then occurs): weights below floor = total * 2^-40
+ * are raised to it.  Plain Huffman: repeatedly merge the two lightest trees (ties: the tree whose
+ * smallest symbol index is lower comes first); a symbol's length is its depth.  If the longest
+ * word exceeds max_len the floor is doubled and the construction repeated (with all weights equal
+ * the depth is ceil(log2 n) <= 8, so this ends).  n = 1 gives length 1.
+ * ---------------------------------------------------------------------------------- */
+int orc_huffman_lengths(const double* w, int n, int max_len, uint8_t* len)
+{
+    if (n < 1 || n > 256 || max_len < 8 || max_len > 32) return 0;
+    if (n == 1) { len[0] = 1; return 1; }
+    double total = 0.0;
+    for (int i = 0; i < n; ++i) { if (!(w[i] >= 0.0)) return 0; total += w[i]; }
+    if (!(total > 0.0)) total = 1.0;
+    double floor_w = total * 9.094947017729282e-13;      /* 2^-40 of the total */
+    for (;;) {
+        double wt[511]; int parent[511]; int lowest[511]; int alive[511];
+        int nodes = n;
+        for (int i = 0; i < n; ++i) { wt[i] = w[i] > floor_w ? w[i] : floor_w; parent[i] = -1; lowest[i] = i; alive[i] = 1; }
+        for (int merges = 0; merges < n - 1; ++merges) {
+            int a = -1, b = -1;                           /* the two lightest live trees, a before b */
+            for (int i = 0; i < nodes; ++i) {
+                if (!alive[i]) continue;
+                if (a < 0 || wt[i] < wt[a] || (wt[i] == wt[a] && lowest[i] < lowest[a])) { b = a; a = i; }
+                else if (b < 0 || wt[i] < wt[b] || (wt[i] == wt[b] && lowest[i] < lowest[b])) b = i;
+            }
+            wt[nodes] = wt[a] + wt[b]; parent[nodes] = -1; alive[nodes] = 1;
+            lowest[nodes] = lowest[a] < lowest[b] ? lowest[a] : lowest[b];
+            parent[a] = nodes; parent[b] = nodes; alive[a] = 0; alive[b] = 0;
+            ++nodes;
+        }
+        int longest = 0;
+        for (int i = 0; i < n; ++i) {
+            int d = 0;
+            for (int v = i; parent[v] >= 0; v = parent[v]) ++d;
+            len[i] = (uint8_t)d;
+            if (d > longest) longest = d;
+        }
+        if (longest <= max_len) return 1;
+        floor_w *= 2.0;
+    }
+}
+
+/* Canonical code words from the lengths: symbols ordered by (length, index); the first word is all
+ * zeros, each next word is the previous plus one, shifted left when the length grows.  Words are
+ * written most significant bit first. */
+void orc_canonical_codes(const uint8_t* len, int n, uint32_t* code)
+{
+    uint32_t next = 0; int prev_len = 0;
+    for (int l = 1; l <= 32; ++l)
+        for (int i = 0; i < n; ++i)
+            if (len[i] == l) {
+                next <<= (l - prev_len);
+                code[i] = next;
+                next += 1; prev_len = l;
+            }
+}
+
+/* Entropy-coded form of one block of up to 1024 coordinates (the blocks of the fixed-width layout).
+ * Stream order: s = 32 * lane + p for lane = 0..31, p = 0..31, which is coordinate
+ * c = 128 * (p / 4) + 4 * lane + p % 4 of the block; coordinates c >= count are left out.  Each
+ * coordinate contributes its level's code word, most significant bit first, then, when the level
+ * index is not 0, one sign bit (appendix: one bit for the sign of each non-zero entry).  Stream bit t
+ * is bit t % 32 of word t / 32.  Returns the number of bits; words must hold 1024 * 33 / 32 entries. */
+static void put_bit(uint32_t* words, int64_t t, unsigned bit)
+{
+    if (bit) words[t / 32] |= (uint32_t)1 << (t % 32);
+}
+
+int64_t orc_entropy_encode_block(const uint8_t* idx, const uint8_t* sign, int count,
+                                 const uint8_t* len, const uint32_t* code, uint32_t* words)
+{
+    int64_t t = 0;
+    memset(words, 0, sizeof(uint32_t) * 1056);
+    for (int s = 0; s < 1024; ++s) {
+        int lane = s / 32, p = s % 32;
+        int c = 128 * (p / 4) + 4 * lane + p % 4;
+        if (c >= count) continue;
+        int l = len[idx[c]];
+        for (int j = l - 1; j >= 0; --j) put_bit(words, t++, (code[idx[c]] >> j) & 1u);
+        if (idx[c] != 0) put_bit(words, t++, sign[c] ? 1u : 0u);
+    }
+    return t;
+}
+
+/* Inverse of the above, reading bit by bit: a word of length l is recognised when the bits read so
+ * far equal the code of a symbol of that length.  Returns the number of bits consumed, or -1 when the
+ * stream holds no valid word. */
+int64_t orc_entropy_decode_block(const uint32_t* words, int count, const uint8_t* len, const uint32_t* code,
+                                 int n, uint8_t* idx, uint8_t* sign)
+{
+    int64_t t = 0;
+    for (int s = 0; s < 1024; ++s) {
+        int lane = s / 32, p = s % 32;
+        int c = 128 * (p / 4) + 4 * lane + p % 4;
+        if (c >= count) continue;
+        uint32_t acc = 0; int l = 0, found = -1;
+        while (found < 0) {
+            if (l >= 32) return -1;
+            acc = (acc << 1) | ((words[t / 32] >> (t % 32)) & 1u); ++t; ++l;
+            for (int i = 0; i < n; ++i) if (len[i] == l && code[i] == acc) { found = i; break; }
+        }
+        idx[c] = (uint8_t)found;
+        sign[c] = 0;
+        if (found != 0) { sign[c] = (uint8_t)((words[t / 32] >> (t % 32)) & 1u); ++t; }
+    }
+    return t;
+}

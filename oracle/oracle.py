@@ -72,6 +72,13 @@ def lib():
         L.orc_level_probabilities.argtypes = [u32p, C.c_int64, f32p, C.c_int, C.c_int64, f32p, C.c_int, C.POINTER(C.c_double)]
         L.orc_expected_code_length.restype = C.c_double
         L.orc_expected_code_length.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_int64, C.POINTER(C.c_double)]
+        L.orc_huffman_lengths.restype = C.c_int
+        L.orc_huffman_lengths.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_int, u8p]
+        L.orc_canonical_codes.argtypes = [u8p, C.c_int, u32p]
+        L.orc_entropy_encode_block.restype = C.c_int64
+        L.orc_entropy_encode_block.argtypes = [u8p, u8p, C.c_int, u8p, u32p, u32p]
+        L.orc_entropy_decode_block.restype = C.c_int64
+        L.orc_entropy_decode_block.argtypes = [u32p, C.c_int, u8p, u32p, C.c_int, u8p, u8p]
         L.orc_alt_rates.argtypes = [C.c_double, C.c_double, C.c_double, f32p, f32p]
         L.orc_sq_norm.restype = C.c_double
         L.orc_sq_norm.argtypes = [f32p, C.c_int64]
@@ -225,6 +232,40 @@ def expected_code_length(p: np.ndarray, d: int):
     p = np.ascontiguousarray(p, np.float64); nz = C.c_double(0)
     bits = lib().orc_expected_code_length(_p(p, C.c_double), p.size, d, C.byref(nz))
     return float(bits), nz.value
+
+
+def huffman_lengths(weights, max_len: int = 12) -> np.ndarray:
+    """Code lengths of a Huffman code for the given symbol weights (every symbol gets a word)."""
+    w = np.ascontiguousarray(weights, np.float64); out = np.zeros(w.size, np.uint8)
+    ok = lib().orc_huffman_lengths(_p(w, C.c_double), w.size, max_len, _p(out, C.c_uint8))
+    assert ok
+    return out
+
+
+def canonical_codes(lengths) -> np.ndarray:
+    l = np.ascontiguousarray(lengths, np.uint8); out = np.zeros(l.size, np.uint32)
+    lib().orc_canonical_codes(_p(l, C.c_uint8), l.size, _p(out, C.c_uint32))
+    return out
+
+
+def entropy_encode_block(idx, sign, lengths, codes):
+    """(words, number of bits) of one block of up to 1024 coordinates."""
+    idx = np.ascontiguousarray(idx, np.uint8); sign = np.ascontiguousarray(sign, np.uint8)
+    l = np.ascontiguousarray(lengths, np.uint8); c = np.ascontiguousarray(codes, np.uint32)
+    words = np.zeros(1056, np.uint32)
+    bits = lib().orc_entropy_encode_block(_p(idx, C.c_uint8), _p(sign, C.c_uint8), idx.size, _p(l, C.c_uint8),
+                                          _p(c, C.c_uint32), _p(words, C.c_uint32))
+    return words[: (bits + 31) // 32].copy(), int(bits)
+
+
+def entropy_decode_block(words, count: int, lengths, codes):
+    """(idx, sign, bits consumed) of one block; bits = -1 when the stream is not valid."""
+    w = np.zeros(1056, np.uint32); w[: len(words)] = words
+    l = np.ascontiguousarray(lengths, np.uint8); c = np.ascontiguousarray(codes, np.uint32)
+    idx = np.zeros(count, np.uint8); sg = np.zeros(count, np.uint8)
+    bits = lib().orc_entropy_decode_block(_p(w, C.c_uint32), count, _p(l, C.c_uint8), _p(c, C.c_uint32), l.size,
+                                          _p(idx, C.c_uint8), _p(sg, C.c_uint8))
+    return idx, sg, int(bits)
 
 
 def alt_rates(lam: float, mu: float, qhat: float):
