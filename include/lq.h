@@ -182,6 +182,40 @@ int lq_level_probabilities(const lq_plan* plan, const uint32_t* hist, const floa
                            int32_t staged, double* probs, void* stream);
 int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* counts, void* stream);
 
+/* Entropy stage on top of the fixed-width message (appendix on the coding framework: with the level
+ * frequencies known or estimated, a Huffman code on the level symbols; one sign bit per non-zero entry).
+ * A layer's code is a list of word lengths, 1..LQ_CODE_MAX_LEN bits, one per level index; the words are the
+ * canonical ones (symbols ordered by length, then index; first word all zeros, each next word the previous
+ * plus one, shifted left where the length grows), sent most significant bit first.  Every layer starts with
+ * the flat code (b bits per index).
+ *   lq_code_build   (host only, no device work): Huffman lengths for the weights (probabilities or counts,
+ *                   e.g. from lq_level_probabilities / lq_symbol_counts); every symbol gets a word, and words
+ *                   longer than LQ_CODE_MAX_LEN are avoided by raising the smallest weights.
+ *   lq_code_set/get: lengths host [n], n = 2^b of the layer; set refuses lengths that violate Kraft's inequality
+ *                   and synchronises the device.
+ * Stream of one worker: the layout's blocks of 1024 coordinates, layer after layer, each starting on a 32-bit
+ * word; inside a block the coordinates in the order s = 32 lane + p (coordinate 128 (p / 4) + 4 lane + p % 4),
+ * padding left out; per coordinate the level's word and, for a non-zero index, the sign bit; stream bit t of a
+ * block is bit t % 32 of its word t / 32.
+ *   lq_entropy_encode: packed dev [K][W] -> stream_words dev [K][capacity_words] and block_offsets dev
+ *                   [K][lq_plan_blocks() + 1] (first word of every block; the last entry is the worker's length in
+ *                   words).  A worker whose stream does not fit keeps its offsets but loses the blocks that do not fit:
+ *                   compare the last offset with capacity_words.  (W words always suffice for the flat code.)
+ *   lq_entropy_decode: the inverse, packed fully overwritten; it equals the encoded message except that the sign
+ *                   bit of a coordinate with level index 0 comes back as 0 (the stream carries no sign there; the
+ *                   decoded value is zero either way).  A stream with no valid word, or a block that runs past
+ *                   its end, sets a flag that lq_entropy_status returns (and clears); nothing faults. */
+#define LQ_CODE_MAX_LEN 12
+int lq_code_build(const double* weights, int32_t n, uint8_t* lengths);
+int lq_code_set(lq_plan* plan, int32_t layer, const uint8_t* lengths, int32_t n);
+int lq_code_get(lq_plan* plan, int32_t layer, uint8_t* lengths, int32_t n);
+int64_t lq_plan_blocks(const lq_plan* plan);        /* blocks of 1024 coordinates per worker, all layers */
+int lq_entropy_encode(lq_plan* plan, const uint32_t* packed, uint32_t* stream_words, int64_t capacity_words,
+                      uint32_t* block_offsets, void* stream);
+int lq_entropy_decode(lq_plan* plan, const uint32_t* stream_words, int64_t capacity_words,
+                      const uint32_t* block_offsets, uint32_t* packed, void* stream);
+int lq_entropy_status(lq_plan* plan, uint32_t* host_flag);
+
 /* Alternative adaptive step sizes (Eq. Alt with the running sums of the appendix on the almost-sure
  * boundedness model): with q_hat in (0, 1/4], every following qoda_step uses
  *   eta_{t+1} = fp32((1 + lambda_{t-1} + mu_{t-1})^(-1/2)),  gamma_{t+1} = fp32((1 + lambda_{t-1})^(q_hat - 1/2)),

@@ -24,7 +24,8 @@ STATUS_NONFINITE = 2
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_norm_scope", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
+           "qoda_get_scalars", "lq_code_build", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
+           "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
@@ -64,6 +65,14 @@ def load_library() -> C.CDLL:
     L.qoda_init.argtypes = [vp, vp, vp, vp, vp]
     L.qoda_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    u8p = C.POINTER(C.c_uint8)
+    L.lq_code_build.argtypes = [C.POINTER(C.c_double), i32, u8p]
+    L.lq_code_set.argtypes = [vp, i32, u8p, i32]
+    L.lq_code_get.argtypes = [vp, i32, u8p, i32]
+    L.lq_plan_blocks.argtypes = [vp]; L.lq_plan_blocks.restype = i64
+    L.lq_entropy_encode.argtypes = [vp, vp, vp, i64, vp, vp]
+    L.lq_entropy_decode.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.lq_entropy_status.argtypes = [vp, C.POINTER(u32)]
     L.lq_level_probabilities.argtypes = [vp, vp, vp, i32, i32, vp, vp]
     L.lq_symbol_counts.argtypes = [vp, vp, vp, vp]
     L.qoda_set_alt_rates.argtypes = [vp, C.c_double]
@@ -109,6 +118,14 @@ def lq_vector_norm_static(v: torch.Tensor, q: int, norm_out: torch.Tensor,
     _check(load_library().lq_vector_norm_static(_ptr(v, torch.float32), v.numel(), int(q),
                                                 _ptr(norm_out, torch.float32), _ptr(status_out, torch.int32),
                                                 _stream()))
+
+
+def lq_code_build(weights) -> List[int]:
+    """Huffman word lengths for the given symbol weights (host only)."""
+    n = len(weights)
+    w = (C.c_double * n)(*[float(x) for x in weights]); out = (C.c_uint8 * n)()
+    _check(load_library().lq_code_build(w, n, out))
+    return list(out)
 
 
 class Plan:
@@ -210,6 +227,33 @@ class Plan:
 
     def lq_symbol_counts(self, packed, counts) -> None:
         _check(load_library().lq_symbol_counts(self._h, _ptr(packed, torch.int32), _ptr(counts, torch.int32), _stream()))
+
+    # ---- entropy stage --------------------------------------------------------------------
+    def lq_code_set(self, layer: int, lengths) -> None:
+        arr = (C.c_uint8 * len(lengths))(*[int(x) for x in lengths])
+        _check(load_library().lq_code_set(self._h, layer, arr, len(lengths)))
+
+    def lq_code_get(self, layer: int) -> List[int]:
+        n = 1 << self.bits[layer]
+        arr = (C.c_uint8 * n)()
+        _check(load_library().lq_code_get(self._h, layer, arr, n))
+        return list(arr)
+
+    def lq_plan_blocks(self) -> int:
+        return int(load_library().lq_plan_blocks(self._h))
+
+    def lq_entropy_encode(self, packed, stream_words, block_offsets) -> None:
+        _check(load_library().lq_entropy_encode(self._h, _ptr(packed, torch.int32), _ptr(stream_words, torch.int32),
+                                                stream_words.shape[1], _ptr(block_offsets, torch.int32), _stream()))
+
+    def lq_entropy_decode(self, stream_words, block_offsets, packed) -> None:
+        _check(load_library().lq_entropy_decode(self._h, _ptr(stream_words, torch.int32), stream_words.shape[1],
+                                                _ptr(block_offsets, torch.int32), _ptr(packed, torch.int32), _stream()))
+
+    def lq_entropy_status(self) -> int:
+        flag = C.c_uint32(0)
+        _check(load_library().lq_entropy_status(self._h, C.byref(flag)))
+        return flag.value
 
     def qoda_set_alt_rates(self, q_hat: float) -> None:
         _check(load_library().qoda_set_alt_rates(self._h, float(q_hat)))

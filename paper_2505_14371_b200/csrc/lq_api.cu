@@ -1,6 +1,7 @@
 // Host side of liblq: the plan object and the extern "C" entry points declared in lq.h.
 // No kernel lives here; this file validates arguments, owns the plan's device tables and
 // enqueues the launchers of the other translation units on the caller's stream.
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -80,6 +81,10 @@ struct lq_plan {
     int32_t* d_member_off = nullptr;       // [L + 1] and [L]: the member lists of lq_fit_levels_shared
     int32_t* d_member_layer = nullptr;
     std::vector<int32_t> h_members;        // host staging of both lists (kept alive for the asynchronous copy)
+    uint32_t* d_code_enc = nullptr;        // [L][256]   entropy stage, allocated at its first use
+    uint16_t* d_code_dec = nullptr;        // [L][4096]
+    uint32_t* d_code_bad = nullptr;        // [1] set by a decode that met an invalid stream
+    std::vector<uint8_t> code_len;         // [L][256] host copy of the word lengths
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
@@ -99,7 +104,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -589,6 +594,121 @@ int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches)
         plan->prof_pool.push_back(r.b);
     }
     plan->prof_recs.clear();
+    return LQ_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+// Uploads the tables of one layer's code.
+int upload_code(lq_plan* plan, int layer, const uint8_t* len, int n)
+{
+    std::vector<uint32_t> code(kMaxLevels, 0), enc(kMaxLevels, 0);
+    std::vector<uint16_t> dec((size_t)1 << kCodeMaxLen);
+    if (!canonical_codes_host(len, n, kCodeMaxLen, code.data()))
+        return fail(LQ_EINVAL, "layer %d: lengths must lie in [1, %d] and satisfy Kraft's inequality", layer, kCodeMaxLen);
+    build_code_tables_host(len, code.data(), n, enc.data(), dec.data());
+    LQ_CUDA(cudaMemcpy(plan->d_code_enc + (size_t)layer * kMaxLevels, enc.data(), kMaxLevels * sizeof(uint32_t),
+                       cudaMemcpyHostToDevice));
+    LQ_CUDA(cudaMemcpy(plan->d_code_dec + ((size_t)layer << kCodeMaxLen), dec.data(), dec.size() * sizeof(uint16_t),
+                       cudaMemcpyHostToDevice));
+    std::copy(len, len + n, plan->code_len.begin() + (size_t)layer * kMaxLevels);
+    return LQ_OK;
+}
+
+// First use of the entropy stage: tables for every layer, initialised to the flat code (b bits per index).
+int ensure_codes(lq_plan* plan)
+{
+    if (plan->d_code_enc) return LQ_OK;
+    const size_t L = (size_t)(plan->dev.num_layers ? plan->dev.num_layers : 1);
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(dev_alloc_zero(&plan->d_code_enc, L * kMaxLevels));
+    LQ_CUDA(dev_alloc_zero(&plan->d_code_dec, L << kCodeMaxLen));
+    LQ_CUDA(dev_alloc_zero(&plan->d_code_bad, 1));
+    try { plan->code_len.assign(L * kMaxLevels, 0); } catch (const std::bad_alloc&) { return fail(LQ_ENOMEM, "host allocation failed"); }
+    for (int m = 0; m < plan->dev.num_layers; ++m) {
+        const LayerDesc& Ld = plan->layers[(size_t)m];
+        uint8_t flat[kMaxLevels];
+        for (int j = 0; j < Ld.nlevels; ++j) flat[j] = (uint8_t)Ld.bits;
+        const int rc = upload_code(plan, m, flat, Ld.nlevels);
+        if (rc != LQ_OK) return rc;
+    }
+    return LQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lq_code_build(const double* weights, int32_t n, uint8_t* lengths)
+{
+    if (!weights || !lengths) return fail(LQ_EINVAL, "NULL argument");
+    if (n < 1 || n > kMaxLevels) return fail(LQ_EINVAL, "n must be in [1, %d]", kMaxLevels);
+    try {
+        if (!huffman_lengths_host(weights, n, kCodeMaxLen, lengths)) return fail(LQ_EINVAL, "weights must be non-negative numbers");
+    } catch (const std::bad_alloc&) { return fail(LQ_ENOMEM, "host allocation failed"); }
+    return LQ_OK;
+}
+
+int lq_code_set(lq_plan* plan, int32_t layer, const uint8_t* lengths, int32_t n)
+{
+    if (!plan || !lengths) return fail(LQ_EINVAL, "NULL argument");
+    if (layer < 0 || layer >= plan->dev.num_layers) return fail(LQ_EINVAL, "layer %d out of range", layer);
+    if (n != plan->layers[(size_t)layer].nlevels) return fail(LQ_EINVAL, "layer %d has %d levels, got %d", layer, plan->layers[(size_t)layer].nlevels, n);
+    const int rc = ensure_codes(plan);
+    if (rc != LQ_OK) return rc;
+    LQ_CUDA(cudaDeviceSynchronize());
+    return upload_code(plan, layer, lengths, n);
+}
+
+int lq_code_get(lq_plan* plan, int32_t layer, uint8_t* lengths, int32_t n)
+{
+    if (!plan || !lengths) return fail(LQ_EINVAL, "NULL argument");
+    if (layer < 0 || layer >= plan->dev.num_layers) return fail(LQ_EINVAL, "layer %d out of range", layer);
+    if (n != plan->layers[(size_t)layer].nlevels) return fail(LQ_EINVAL, "layer %d has %d levels, got %d", layer, plan->layers[(size_t)layer].nlevels, n);
+    const int rc = ensure_codes(plan);
+    if (rc != LQ_OK) return rc;
+    std::copy(plan->code_len.begin() + (size_t)layer * kMaxLevels, plan->code_len.begin() + (size_t)layer * kMaxLevels + n, lengths);
+    return LQ_OK;
+}
+
+int64_t lq_plan_blocks(const lq_plan* plan) { return plan ? plan->dev.total_blocks : (int64_t)fail(LQ_EINVAL, "plan is NULL"); }
+
+int lq_entropy_encode(lq_plan* plan, const uint32_t* packed, uint32_t* stream_words, int64_t capacity_words,
+                      uint32_t* block_offsets, void* stream)
+{
+    if (!plan || !packed || !stream_words || !block_offsets) return fail(LQ_EINVAL, "NULL argument");
+    if (capacity_words < 0) return fail(LQ_EINVAL, "capacity_words < 0");
+    LQ_ALIGNED(packed, 4); LQ_ALIGNED(stream_words, 4); LQ_ALIGNED(block_offsets, 4);
+    const int rc = ensure_codes(plan);
+    if (rc != LQ_OK) return rc;
+    LQ_CUDA(launch_entropy_encode(plan->dev, packed, plan->d_code_enc, block_offsets, stream_words, capacity_words,
+                                  (cudaStream_t)stream));
+    return LQ_OK;
+}
+
+int lq_entropy_decode(lq_plan* plan, const uint32_t* stream_words, int64_t capacity_words,
+                      const uint32_t* block_offsets, uint32_t* packed, void* stream)
+{
+    if (!plan || !packed || !stream_words || !block_offsets) return fail(LQ_EINVAL, "NULL argument");
+    if (capacity_words < 0) return fail(LQ_EINVAL, "capacity_words < 0");
+    LQ_ALIGNED(packed, 4); LQ_ALIGNED(stream_words, 4); LQ_ALIGNED(block_offsets, 4);
+    const int rc = ensure_codes(plan);
+    if (rc != LQ_OK) return rc;
+    LQ_CUDA(launch_entropy_decode(plan->dev, stream_words, capacity_words, block_offsets, plan->d_code_dec, packed,
+                                  plan->d_code_bad, (cudaStream_t)stream));
+    return LQ_OK;
+}
+
+int lq_entropy_status(lq_plan* plan, uint32_t* host_flag)
+{
+    if (!plan || !host_flag) return fail(LQ_EINVAL, "NULL argument");
+    *host_flag = 0;
+    if (!plan->d_code_bad) return LQ_OK;
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(host_flag, plan->d_code_bad, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    LQ_CUDA(cudaMemset(plan->d_code_bad, 0, sizeof(uint32_t)));
     return LQ_OK;
 }
 

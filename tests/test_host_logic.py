@@ -101,3 +101,29 @@ def test_reference_arm_runs_on_rank_zero_only():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],
                          capture_output=True, text=True, timeout=120, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_library_code_builder_is_optimal_like_the_oracles(orc):
+    """lq_code_build runs on the host only.  Huffman lengths are not unique under ties, so the two builders are
+    compared through what is unique: the expected length (optimal), Kraft's equality and the length limit."""
+    import numpy as np
+    from paper_2505_14371_b200 import binding
+    binding.load_library()
+    rng = np.random.default_rng(12)
+    for n in (1, 2, 4, 8, 16, 32, 256):
+        for _ in range(5):
+            w = rng.dirichlet(np.ones(n) * 0.3) if n > 1 else np.ones(1)
+            if n > 2:
+                w[rng.integers(0, n)] = 0.0
+            ours = np.array(binding.lq_code_build(w))
+            ref = orc.huffman_lengths(w).astype(int)
+            assert ours.min() >= 1 and ours.max() <= 12
+            if n > 1:
+                assert abs(sum(2.0 ** -int(x) for x in ours) - 1.0) < 1e-12
+            wf = np.maximum(w, w.sum() * 2.0 ** -40)
+            assert abs(float((wf * ours).sum()) - float((wf * ref).sum())) <= 1e-9 * float((wf * ref).sum())
+    geometric = 0.5 ** np.arange(40)
+    assert max(binding.lq_code_build(geometric)) == 12
+    assert binding.lq_code_build([0.4, 0.3, 0.2, 0.1]) == [1, 2, 3, 3]
+    with pytest.raises(binding.LqError):
+        binding.lq_code_build([0.5, -0.1])
