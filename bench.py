@@ -67,6 +67,8 @@ def pick_workload(name: str):
         return W.transformer_xl_workload(num_blocks=2, vocab=8192)
     if name == "transformer_xl_medium":                # all 16 blocks, a quarter of the vocabulary
         return W.transformer_xl_workload(num_blocks=16, vocab=65536)
+    if name.startswith("powersgd:"):                   # powersgd:<rank>: low-rank factor shapes (Section 7.2)
+        return W.powersgd_factor_workload(int(name.split(":")[1]))
     if name.startswith("flat:"):                       # flat:<log2 n>:<bits>:<K>:<q>
         n, b, k, q = (int(x) for x in name.split(":")[1:5])
         return W.flat_workload(n, b, k, q)

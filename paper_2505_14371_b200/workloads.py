@@ -86,6 +86,26 @@ def transformer_xl_workload(num_blocks: int = 16, vocab: int = 267735) -> Worklo
                     zero_row_layers={0: (dm, 0.9)}, config_id=4)
 
 
+def powersgd_factor_workload(rank: int = 32, num_blocks: int = 16, vocab: int = 267735) -> Workload:
+    """Low-rank factor shapes of the Transformer-XL experiment (Section 7.2): every weight matrix (n x m) of the
+    model is replaced by its two rank-`rank` factors (n x rank and m x rank), which is what gets quantized
+    there; vectors (biases, LayerNorm) stay as they are.  A factor row is zero where the matrix row is, so
+    the embedding's first factor keeps 90 % zero rows, now `rank` values long."""
+    dm, nh, dh, dff = 410, 10, 41, 2100
+    mats = [(vocab, dm)]
+    vecs: List[int] = []
+    for _ in range(num_blocks):
+        mats += [(dm, 3 * nh * dh), (dm, dm), (dm, dm), (dm, dff), (dff, dm)]
+        vecs += [3 * nh * dh, dm, dm, dff, dm, dm, dm, dm, dm]
+    sizes: List[int] = []
+    for n, m in mats:
+        sizes += [n * rank, m * rank]
+    sizes += vecs
+    return Workload(f"powersgd_rank{rank}", sizes, bits=4, q=2, num_workers=8, dist="normal",
+                    scales=_log_uniform_scales(len(sizes), -4.0, -1.0, SEED_BASE + 6),
+                    zero_row_layers={0: (rank, 0.9)}, config_id=6)
+
+
 def flat_workload(log2_n: int, bits: int, num_workers: int, q: int) -> Workload:
     """Config 5a: one flat N(0,1) layer of 2**log2_n coordinates."""
     return Workload(f"flat_2^{log2_n}", [1 << log2_n], bits=bits, q=q,

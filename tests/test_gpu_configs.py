@@ -149,6 +149,32 @@ def test_config3_wgan_full_size_element_by_element(lqm, orc):
     assert t == 3 and abs(S - model.S) <= 1e-9 * model.S and abs(eta - float(model.eta)) <= 1e-6 * eta
 
 
+def test_low_rank_factor_shapes_two_iterations(lqm, orc):
+    """The rank-16 factor shapes of the Section 7.2 model (2 blocks, 8192-row embedding: 37 layers from 410 to
+    131 072 coordinates, zero rows 16 values long): two iterations against the oracle, everything bit-exact."""
+    from paper_2505_14371_b200 import workloads as W
+    w = W.powersgd_factor_workload(rank=16, num_blocks=2, vocab=8192)
+    K = w.num_workers
+    plan = lqm.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda")
+    model = oracle_model(orc, plan)
+    X1 = torch.zeros(plan.padded_elems, device="cuda"); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    gbar = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh); model.qoda_init(to_unpadded(plan, X1))
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    for t in (1, 2):
+        c, p = t % 2, (t + 1) % 2
+        gt = grads if t == 1 else torch.roll(grads, 1, dims=0) * 0.7
+        plan.lq_quantize_pack(gt, t, pk[c], nm[c], prev_packed=pk[p] if t > 1 else None,
+                              prev_norms=nm[p] if t > 1 else None)
+        plan.qoda_step(pk[c], nm[c], X1, Y, Xh, None, gbar)
+        ref = model.quantize(to_unpadded(plan, gt), t)
+        assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+        assert np.array_equal(nm[c].cpu().numpy()[:, :plan.num_layers], ref["norms"])
+        assert np.array_equal(to_unpadded(plan, gbar), model.qoda_step())
+        assert _rel(to_unpadded(plan, Y), model.Y) <= 1e-6 and _rel(to_unpadded(plan, Xh), model.Xhalf) <= 1e-6
+
+
 # ------------------------------------------------------------------------------ config 4
 def test_config4_transformer_xl_full_size_sampled(lqm, orc):
     """The benchmark's workload and launch configuration (150 870 550 coordinates x K = 8, 4 bits): sampled
