@@ -85,7 +85,30 @@ int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, in
  * Takes effect at the next lq_layer_norms / lq_quantize_pack. */
 #define LQ_NORM_PER_LAYER 0
 #define LQ_NORM_GLOBAL    1
+/* LQ_NORM_BUCKET: the setting of the experiments in Section 7.1 - every bucket of LQ_BUCKET = 128 consecutive
+ * coordinates of a layer (the last one of a layer may be shorter) is normalised by its own L^q norm, with the
+ * layer's level sequence.  Differences from the other scopes:
+ *  - a norms buffer is [K][lq_plan_norm_count()] fp32: for layer m, block i of 1024 coordinates and row j of 128,
+ *    the bucket's norm sits at 8 * (blocks of the layers before m + i) + j; rows past the layer's end hold 0.
+ *    lq_quantize_pack WRITES it in its single pass over the values (there is no separate norm pass and
+ *    lq_layer_norms is refused); prev_norms, lq_decode_aggregate and qoda_step read the same shape;
+ *  - a bucket that is all zero, whose norm is below the smallest normal float, or that holds NaN or Inf has norm
+ *    0 and sends zeros; the layer's flag (lq_get_statistics) is LQ_STATUS_NONFINITE if any of its buckets held NaN
+ *    or Inf, else LQ_STATUS_ZERO_NORM if none of its buckets has a nonzero norm;
+ *  - the histogram of a (worker, layer) pools its buckets' normalised magnitudes (zeroed buckets add nothing);
+ *    lq_fit_levels, lq_fit_levels_shared and lq_level_probabilities weight worker k's histogram of layer m by
+ *    the layer's energy, the sum of its squared bucket norms as left by the plan's last lq_quantize_pack
+ *    (lq_layer_weights returns its square root), and do not read their `norms` argument (any non-NULL pointer).
+ * The bucket scope can only be entered or left before the plan's first lq_quantize_pack (else LQ_ESTATE). */
+#define LQ_NORM_BUCKET    2
+#define LQ_BUCKET         128
 int lq_set_norm_scope(lq_plan* plan, int32_t scope);
+/* fp32 values per worker in a norms buffer under the plan's current scope: the number of layers, or in bucket
+ * scope 8 x the number of 1024-coordinate blocks of all layers.  Negative error code on failure. */
+int64_t lq_plan_norm_count(const lq_plan* plan);
+/* Bucket scope: host_weights [K][L] receives sqrt(sum of squared bucket norms) of every (worker, layer) of the
+ * plan's last lq_quantize_pack.  Synchronises the device.  LQ_ESTATE in another scope. */
+int lq_layer_weights(const lq_plan* plan, float* host_weights);
 
 /* Level sequence of one layer (Section 3.1: 0 = l_0 < l_1 < ... < l_{n-1} = 1, n = 2^b).
  * host_levels [n] host.  set: validates (n must equal 2^b, increasing by at least 2^-100 per

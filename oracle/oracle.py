@@ -312,6 +312,7 @@ class OracleModel:
         self.prev_decoded = None         # [K][D] decoded V^_{k,t-1/2}
         self.pending_sq = None
         self.norm_scope = "layer"        # "global": one norm over the worker's whole vector (Section 3.1, definition of Q)
+                                         # "bucket": one norm per 128 consecutive coordinates of a layer (Section 7.1)
         self.alt_qhat = 0.0              # > 0: the alternative rates of Eq. (Alt) with this exponent
         self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
 
@@ -328,6 +329,8 @@ class OracleModel:
         decoded = np.zeros((K, self.D), np.float32)
         sq = np.zeros((K, Lr), np.float64)
         near = 0
+        if self.norm_scope == "bucket":
+            return self._quantize_bucketed(grads, step, want_hist)
         for k in range(K):
             if self.norm_scope == "global":      # ||v||_q of the whole vector, shared by every layer of the worker
                 gn, gs = layer_norm(grads[k], self.q)
@@ -350,6 +353,50 @@ class OracleModel:
         self.pending_sq = sq
         self.cur_decoded = decoded
         return dict(norms=norms, status=status, idx=idx, sign=sg, packed=packed, hist=hist,
+                    near=near, sq_diff=sq, decoded=decoded)
+
+    def _quantize_bucketed(self, grads: np.ndarray, step: int, want_hist: bool, bucket: int = 128):
+        """The quantizer applied bucket by bucket (Section 7.1: buckets of 128 coordinates): every bucket of a layer
+        is a vector of its own with its own norm and the layer's level sequence; coordinate indices (the random
+        numbers' counters) stay those of the layer.  A layer's histogram pools its buckets; its weight in the
+        level fit is the square root of the summed squared bucket norms; status 2 if any bucket held NaN or Inf,
+        else 1 if no bucket has a nonzero norm."""
+        K, Lr = self.K, len(self.sizes)
+        status = np.zeros((K, Lr), np.int32); weights = np.zeros((K, Lr), np.float32)
+        bnorms = [[None] * Lr for _ in range(K)]
+        idx = np.zeros((K, self.D), np.uint8); sg = np.zeros((K, self.D), np.uint8)
+        packed = [[None] * Lr for _ in range(K)]
+        hist = np.zeros((K, Lr, HIST_STRIDE), np.uint32) if want_hist else None
+        decoded = np.zeros((K, self.D), np.float32)
+        sq = np.zeros((K, Lr), np.float64)
+        near = 0
+        for k in range(K):
+            for m in range(Lr):
+                a, b = int(self.off[m]), int(self.off[m + 1])
+                nb = (b - a + bucket - 1) // bucket
+                bn = np.zeros(nb, np.float32)
+                any_bad, any_live, energy = False, False, 0.0
+                for i in range(nb):
+                    lo, hi = a + i * bucket, min(a + (i + 1) * bucket, b)
+                    v = grads[k, lo:hi]
+                    bn[i], st = layer_norm(v, self.q)
+                    any_bad |= st == 2; any_live |= bn[i] > 0
+                    energy += float(bn[i]) * float(bn[i])
+                    i_, s_, nr = quantize_layer(v, bn[i], self.levels[m], self.seed, step, k, m, first_index=lo - a)
+                    near += nr
+                    idx[k, lo:hi], sg[k, lo:hi] = i_, s_
+                    if want_hist:
+                        hist[k, m] += histogram_layer(v, bn[i])
+                    decoded[k, lo:hi] = decode_layer(i_, s_, bn[i], self.levels[m])
+                bnorms[k][m] = bn
+                weights[k, m] = np.float32(np.sqrt(energy))
+                status[k, m] = 2 if any_bad else (0 if any_live else 1)
+                packed[k][m] = pack_layer(idx[k, a:b], sg[k, a:b], self.bits[m])
+                prev = None if self.prev_decoded is None else self.prev_decoded[k, a:b]
+                sq[k, m] = sq_diff(decoded[k, a:b], prev)
+        self.pending_sq = sq
+        self.cur_decoded = decoded
+        return dict(norms=weights, bucket_norms=bnorms, status=status, idx=idx, sign=sg, packed=packed, hist=hist,
                     near=near, sq_diff=sq, decoded=decoded)
 
     def fit(self, hist: np.ndarray, norms: np.ndarray) -> None:

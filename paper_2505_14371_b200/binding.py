@@ -22,7 +22,7 @@ STATUS_ZERO_NORM = 1
 STATUS_NONFINITE = 2
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
-           "lq_plan_layer_info", "lq_set_norm_scope", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
+           "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_code_build", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
            "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
@@ -55,6 +55,9 @@ def load_library() -> C.CDLL:
     L.lq_plan_packed_words.argtypes = [vp]; L.lq_plan_packed_words.restype = i64
     L.lq_plan_layer_info.argtypes = [vp, i32, C.POINTER(i64), C.POINTER(i64), C.POINTER(i32)]
     L.lq_set_norm_scope.argtypes = [vp, i32]
+    L.lq_plan_norm_count.argtypes = [vp]
+    L.lq_plan_norm_count.restype = i64
+    L.lq_layer_weights.argtypes = [vp, vp]
     L.lq_set_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_get_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_layer_norms.argtypes = [vp, vp, vp, vp]
@@ -166,8 +169,20 @@ class Plan:
             pass
 
     def lq_set_norm_scope(self, scope: str) -> None:
-        """"layer" (default) or "global" (one norm over the worker's whole vector)."""
-        _check(load_library().lq_set_norm_scope(self._h, {"layer": 0, "global": 1}[scope]))
+        """"layer" (default), "global" (one norm over the worker's whole vector) or "bucket" (one norm per 128
+        consecutive coordinates of a layer; norms buffers then have lq_plan_norm_count() values per worker)."""
+        _check(load_library().lq_set_norm_scope(self._h, {"layer": 0, "global": 1, "bucket": 2}[scope]))
+
+    def lq_plan_norm_count(self) -> int:
+        n = int(load_library().lq_plan_norm_count(self._h))
+        if n < 0:
+            _check(n)
+        return n
+
+    def lq_layer_weights(self) -> torch.Tensor:
+        out = torch.empty((self.num_workers, max(self.num_layers, 1)), dtype=torch.float32)
+        _check(load_library().lq_layer_weights(self._h, out.data_ptr()))
+        return out[:, :self.num_layers]
 
     # ---- levels -------------------------------------------------------------------------
     def lq_set_levels(self, layer: int, levels) -> None:
@@ -286,7 +301,7 @@ class Plan:
         return torch.empty((self.num_workers, max(self.packed_words, 1)), dtype=torch.int32, device=device)
 
     def empty_norms(self, device="cuda") -> torch.Tensor:
-        return torch.empty((self.num_workers, max(self.num_layers, 1)), dtype=torch.float32, device=device)
+        return torch.empty((self.num_workers, max(self.lq_plan_norm_count(), 1)), dtype=torch.float32, device=device)
 
     def zero_hist(self, device="cuda") -> torch.Tensor:
         return torch.zeros((self.num_workers, max(self.num_layers, 1), HIST_STRIDE), dtype=torch.int32,

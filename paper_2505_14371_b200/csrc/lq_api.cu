@@ -105,6 +105,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
     cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.energy_partial); cudaFree(p->dev.flag_partial); cudaFree(p->dev.layer_weight);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
     delete p;
@@ -241,6 +242,9 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_total, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.energy_partial, KT);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.flag_partial, KT);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_weight, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_member_off, nl + 1);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_member_layer, nl);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.alt_partial, 2 * (size_t)(ntiles ? ntiles : 1) * (size_t)d.sub_tiles);
@@ -342,6 +346,8 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
 {
     if (!plan || !grads || !norms) return fail(LQ_EINVAL, "NULL argument");
     LQ_ALIGNED(grads, 16); LQ_ALIGNED(norms, 4);
+    if (plan->dev.bucket_norm)
+        return fail(LQ_EINVAL, "lq_layer_norms: in bucket scope the norms are written by lq_quantize_pack");
     if (plan->dev.num_layers == 0) return LQ_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const PlanDev& d = plan->dev;
@@ -380,6 +386,16 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     const PlanDev& d = plan->dev;
     const float* lc = plan->d_levels_enc[plan->cur];
     const float* lp = plan->d_levels_enc[plan->prev];
+    if (d.bucket_norm) {                 // one pass: the norms come out of the encoder itself
+        LQ_CUDA(timed(plan, LQ_KERNEL_QUANTIZE_PACK, s, [&] {
+            return launch_quantize_bucketed(d, grads, step, packed, norms, hist, prev_packed, prev_norms, lc, lp,
+                                            plan->search, s);
+        }));
+        LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_bucket_finalize(d, s); }));
+        plan->have_message = true;
+        plan->stat_pending = true;
+        return LQ_OK;
+    }
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, true, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_QUANTIZE_PACK, s, [&] {
@@ -399,7 +415,8 @@ int lq_fit_levels(lq_plan* plan, const uint32_t* hist, const float* norms, int32
         return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
     cudaStream_t s = (cudaStream_t)stream;
     LQ_CUDA(timed(plan, LQ_KERNEL_FIT, s, [&] {
-        return launch_fit(plan->dev, hist, norms, num_samples, plan->d_levels_stage, s);
+        return launch_fit(plan->dev, hist, plan->dev.bucket_norm ? plan->dev.layer_weight : norms, num_samples,
+                          plan->d_levels_stage, s);
     }));
     plan->stage_dirty = true;
     return LQ_OK;
@@ -444,7 +461,8 @@ int lq_fit_levels_shared(lq_plan* plan, const uint32_t* hist, const float* norms
     LQ_CUDA(cudaMemcpyAsync(plan->d_member_layer, plan->h_members.data() + off.size(), members.size() * sizeof(int32_t),
                             cudaMemcpyHostToDevice, s));
     LQ_CUDA(timed(plan, LQ_KERNEL_FIT, s, [&] {
-        return launch_fit_shared(plan->dev, hist, norms, num_samples, plan->d_levels_stage, plan->d_member_off,
+        return launch_fit_shared(plan->dev, hist, plan->dev.bucket_norm ? plan->dev.layer_weight : norms, num_samples,
+                                 plan->d_levels_stage, plan->d_member_off,
                                  plan->d_member_layer, num_types, s);
     }));
     plan->stage_dirty = true;
@@ -505,8 +523,29 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
 int lq_set_norm_scope(lq_plan* plan, int32_t scope)
 {
     if (!plan) return fail(LQ_EINVAL, "plan is NULL");
-    if (scope != LQ_NORM_PER_LAYER && scope != LQ_NORM_GLOBAL) return fail(LQ_EINVAL, "unknown norm scope %d", scope);
+    if (scope != LQ_NORM_PER_LAYER && scope != LQ_NORM_GLOBAL && scope != LQ_NORM_BUCKET)
+        return fail(LQ_EINVAL, "unknown norm scope %d", scope);
+    const int bucket = scope == LQ_NORM_BUCKET ? 1 : 0;
+    if (bucket != plan->dev.bucket_norm && plan->have_message)
+        return fail(LQ_ESTATE, "the bucket scope can only be entered or left before the first lq_quantize_pack");
     plan->dev.global_norm = scope == LQ_NORM_GLOBAL ? 1 : 0;
+    plan->dev.bucket_norm = bucket;
+    return LQ_OK;
+}
+
+int64_t lq_plan_norm_count(const lq_plan* plan)
+{
+    if (!plan) return (int64_t)fail(LQ_EINVAL, "plan is NULL");
+    return plan->dev.bucket_norm ? plan->dev.total_blocks * 8 : (int64_t)plan->dev.num_layers;
+}
+
+int lq_layer_weights(const lq_plan* plan, float* host_weights)
+{
+    if (!plan || !host_weights) return fail(LQ_EINVAL, "NULL argument");
+    if (!plan->dev.bucket_norm) return fail(LQ_ESTATE, "lq_layer_weights: the plan is not in bucket scope");
+    LQ_CUDA(cudaDeviceSynchronize());
+    LQ_CUDA(cudaMemcpy(host_weights, plan->dev.layer_weight,
+                       (size_t)plan->dev.num_workers * (size_t)plan->dev.num_layers * sizeof(float), cudaMemcpyDeviceToHost));
     return LQ_OK;
 }
 
@@ -517,7 +556,8 @@ int lq_level_probabilities(const lq_plan* plan, const uint32_t* hist, const floa
     if (num_samples < 1 || num_samples > LQ_MAX_WORKERS)
         return fail(LQ_EINVAL, "num_samples must be in [1, %d]", LQ_MAX_WORKERS);
     const float* levels = staged ? plan->d_levels_stage : plan->d_levels_enc[plan->cur];
-    LQ_CUDA(launch_level_probabilities(plan->dev, hist, norms, num_samples, levels, probs, (cudaStream_t)stream));
+    LQ_CUDA(launch_level_probabilities(plan->dev, hist, plan->dev.bucket_norm ? plan->dev.layer_weight : norms,
+                                       num_samples, levels, probs, (cudaStream_t)stream));
     return LQ_OK;
 }
 

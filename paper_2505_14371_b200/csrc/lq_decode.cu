@@ -27,11 +27,13 @@ constexpr int kStageBytes = kWarps * 2 * kPartRows * 512;   // per CTA: each war
 // string holds its symbols 16 H .. 16 H + 15 (rows 4 H .. 4 H + 3 of the block); only the words that
 // carry those symbols are read.  All workers' words are requested before the first one is used, so
 // that a warp keeps a few KB in flight.  `table[kk]` holds N * l_j at 2j and -N * l_j at 2j + 1 for
-// worker kk of the chunk.
-template <int B, int H>
+// worker kk of the chunk.  Bucket scope: table[0] holds the plain signed levels for every worker, and `bn` points
+// at worker k0's norms of this piece's rows (one per row of 128 coordinates; the next worker's `bn_stride` further).
+template <int B, int H, bool kBucket>
 __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const uint32_t* __restrict__ words,
                                                   int64_t worker_stride, int kc,
-                                                  const float (*table)[2 * kMaxLevels])
+                                                  const float (*table)[2 * kMaxLevels],
+                                                  const float* __restrict__ bn, int64_t bn_stride)
 {
     constexpr int C = B + 1;
     constexpr int kFirst = (kPartSyms * H * C) >> 5;                  // first and last word of this piece
@@ -42,13 +44,22 @@ __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const
 #pragma unroll
         for (int i = 0; i < C; ++i)
             w[kk][i] = (i >= kFirst && i <= kLast && kk < kc) ? __ldcs(words + kk * worker_stride + i * 32) : 0u;
+    float nr[kBucket ? kWorkerChunk : 1][kPartRows];
+    if (kBucket) {
+#pragma unroll
+        for (int kk = 0; kk < kWorkerChunk; ++kk)
+#pragma unroll
+            for (int jj = 0; jj < kPartRows; ++jj) nr[kk][jj] = kk < kc ? __ldg(bn + kk * bn_stride + jj) : 0.0f;
+    }
 #pragma unroll
     for (int kk = 0; kk < kWorkerChunk; ++kk) {
         if (kk < kc) {
-            const char* tb = reinterpret_cast<const char*>(table[kk]);
+            const char* tb = reinterpret_cast<const char*>(table[kBucket ? 0 : kk]);
 #pragma unroll
-            for (int p = 0; p < kPartSyms; ++p)
-                acc[p] += *reinterpret_cast<const float*>(tb + symbol4_at<C>(w[kk], kPartSyms * H + p));
+            for (int p = 0; p < kPartSyms; ++p) {
+                const float val = *reinterpret_cast<const float*>(tb + symbol4_at<C>(w[kk], kPartSyms * H + p));
+                acc[p] += kBucket ? __fmul_rn(val, nr[kk][p >> 2]) : val;
+            }
         }
     }
 }
@@ -67,15 +78,17 @@ struct DecodeArgs {
     float* gbar;
 };
 
-// Fills the value tables of workers k0 .. k0 + kc - 1 of one layer (CTA-wide, between two barriers).
+// Fills the value tables of workers k0 .. k0 + kc - 1 of one layer (CTA-wide, between two barriers); in bucket
+// scope one table of plain signed levels.
+template <bool kBucket>
 __device__ __forceinline__ void fill_tables(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
                                             float (*table)[2 * kMaxLevels], int k0, int kc)
 {
     __syncthreads();
-    for (int i = threadIdx.x; i < kc * L.nlevels; i += blockDim.x) {
+    for (int i = threadIdx.x; i < (kBucket ? 1 : kc) * L.nlevels; i += blockDim.x) {
         const int kk = i / L.nlevels, j = i - kk * L.nlevels;
-        const float mag = __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer],
-                                    a.levels[(int64_t)layer * kLevelStride + j]);
+        const float lv = a.levels[(int64_t)layer * kLevelStride + j];
+        const float mag = kBucket ? lv : __fmul_rn(a.norms[(int64_t)(k0 + kk) * p.num_layers + layer], lv);
         table[kk][2 * j] = mag;                       // symbol = 2 * idx + sign
         table[kk][2 * j + 1] = -mag;
     }
@@ -85,7 +98,7 @@ __device__ __forceinline__ void fill_tables(const PlanDev& p, const LayerDesc& L
 // One half block: the mean of the K decoded messages for rows 4 H .. 4 H + 3, then the update.
 // Any worker count: the accumulators live across chunks of kWorkerChunk workers; with a single chunk
 // the tables are filled once per CTA (`resident`).
-template <int B, int H, int kMode>
+template <int B, int H, int kMode, bool kBucket>
 __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
                                             float (*table)[2 * kMaxLevels], const Rates& rt, float invK,
                                             int64_t blk, bool active, bool& resident, float4* stage,
@@ -117,9 +130,12 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     for (int i = 0; i < kPartSyms; ++i) acc[i] = 0.0f;
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
         const int kc = min(kWorkerChunk, K - k0);
-        if (!resident) fill_tables(p, L, layer, a, table, k0, kc);
-        if (K <= kWorkerChunk) resident = true;
-        if (active) decode_accumulate<B, H>(acc, a.packed + (int64_t)k0 * p.packed_words + woff, p.packed_words, kc, table);
+        if (!resident) fill_tables<kBucket>(p, L, layer, a, table, k0, kc);
+        if (kBucket || K <= kWorkerChunk) resident = true;
+        const int64_t bn_stride = p.total_blocks * 8;
+        const float* bn = kBucket ? a.norms + (int64_t)k0 * bn_stride + (L.block_off + blk) * 8 + kPartRows * H : nullptr;
+        if (active) decode_accumulate<B, H, kBucket>(acc, a.packed + (int64_t)k0 * p.packed_words + woff, p.packed_words,
+                                                     kc, table, bn, bn_stride);
     }
     if (!active) return;
     if (kQoda) cp_async_wait<0>();
@@ -165,7 +181,7 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     }
 }
 
-template <int B, int kMode>
+template <int B, int kMode, bool kBucket>
 __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const LayerDesc& L, int layer,
                                                      const Tile& tile, const DecodeArgs& a,
                                                      float (*table)[2 * kMaxLevels], const Rates& rt,
@@ -181,17 +197,17 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
     for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
         const bool active = b0 + warp < tile.nblocks;
         const int64_t blk = tile.block0 + b0 + warp;
-        decode_half<B, 0, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
-        decode_half<B, 1, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+        decode_half<B, 0, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+        decode_half<B, 1, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
         if (kParts == 4) {
-            decode_half<B, 2 % kParts, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
-            decode_half<B, 3 % kParts, kMode>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+            decode_half<B, 2 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+            decode_half<B, 3 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
         }
     }
 }
 
-template <int kMode>
-__global__ void __launch_bounds__(kThreads, kMode == 2 ? 3 : LQ_DEC_CTAS) decode_kernel(PlanDev p, DecodeArgs a)
+template <int kMode, bool kBucket>
+__global__ void __launch_bounds__(kThreads, kBucket ? 2 : (kMode == 2 ? 3 : LQ_DEC_CTAS)) decode_kernel(PlanDev p, DecodeArgs a)
 {
     __shared__ float table[kWorkerChunk][2 * kMaxLevels];
     constexpr bool kAlt = kMode == 2;
@@ -215,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, kMode == 2 ? 3 : LQ_DEC_CTAS) decode
     double lam_acc = 0.0, mu_acc = 0.0;
 
     switch (L.bits) {
-#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kMode>(p, L, layer, tile, a, table, rt, lam_acc, mu_acc); break;
+#define LQ_CASE(BB) case BB: decode_block_chunked<BB, kMode, kBucket>(p, L, layer, tile, a, table, rt, lam_acc, mu_acc); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
@@ -297,9 +313,15 @@ cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float*
     if (p.num_tiles == 0) return cudaSuccess;
     DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
     const unsigned grid = (unsigned)p.num_tiles * p.sub_tiles;
-    if (mode == 2)      decode_kernel<2><<<grid, kThreads, kStageBytes, s>>>(p, a);
-    else if (mode == 1) decode_kernel<1><<<grid, kThreads, kStageBytes, s>>>(p, a);
-    else                decode_kernel<0><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    if (p.bucket_norm) {
+        if (mode == 2)      decode_kernel<2, true><<<grid, kThreads, kStageBytes, s>>>(p, a);
+        else if (mode == 1) decode_kernel<1, true><<<grid, kThreads, kStageBytes, s>>>(p, a);
+        else                decode_kernel<0, true><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    } else {
+        if (mode == 2)      decode_kernel<2, false><<<grid, kThreads, kStageBytes, s>>>(p, a);
+        else if (mode == 1) decode_kernel<1, false><<<grid, kThreads, kStageBytes, s>>>(p, a);
+        else                decode_kernel<0, false><<<grid, kThreads, kStageBytes, s>>>(p, a);
+    }
     return cudaGetLastError();
 }
 

@@ -63,6 +63,7 @@ struct PlanDev {
     int32_t sub_tiles;    // sub-tiles per tile: the plan's tile size / kSubBlocks (1, 2 or 4)
     int32_t sub_shift;    // log2(sub_tiles)
     int32_t global_norm;  // 1: one norm per worker over all layers (Section 3.1), 0: one per layer
+    int32_t bucket_norm;  // 1: one norm per bucket of 128 consecutive coordinates of a layer (Section 7.1)
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;
@@ -76,6 +77,9 @@ struct PlanDev {
     uint8_t* row_mask;    // [K][total_blocks]  bit j of a block's byte: row j (128 values) holds a nonzero value
     const uint8_t* row_mask_prev;   // the same for the input behind the previous message, or NULL when unknown
     int64_t total_blocks; // blocks of 1024 values per worker, all layers
+    double* energy_partial;   // [K][num_tiles]  bucket scope: per-tile sums of squared bucket norms
+    uint32_t* flag_partial;   // [K][num_tiles]  bucket scope: bit 0 a non-finite bucket, bit 1 a nonzero bucket
+    float* layer_weight;      // [K][L]          bucket scope: sqrt of a layer's summed squared bucket norms
     QodaScalars* scalars;
 };
 
@@ -97,6 +101,12 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
                             const float* norms, uint32_t* hist, const uint32_t* prev_packed,
                             const float* prev_norms, const float* levels_cur,
                             const float* levels_prev, SearchTables t, cudaStream_t s);
+// bucket scope: `bucket_norms` [K][8 * total_blocks] is written, `prev_norms` has the same shape
+cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
+                                     float* bucket_norms, uint32_t* hist, const uint32_t* prev_packed,
+                                     const float* prev_norms, const float* levels_cur,
+                                     const float* levels_prev, SearchTables t, cudaStream_t s);
+cudaError_t launch_bucket_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s);
 // mode 0: decode + aggregate only; 1: + QODA update, Eq. (general_stepsize); 2: + QODA update, Eq. (Alt)
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,

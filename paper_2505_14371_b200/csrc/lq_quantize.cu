@@ -163,20 +163,135 @@ __device__ __forceinline__ void issue_ragged_block(const WarpCtx& c, int64_t blk
     }
 }
 
+// Bucket scope (Section 7.1 runs the quantizer on buckets of 128 consecutive coordinates, each with its own
+// norm): a bucket is one row of a block, which a warp holds as one float4 per lane, so the norm is a reduction
+// over the warp and the separate norm pass disappears.
+struct BucketCtx {
+    const float* prev_bn;        // bucket norms of the previous message for this (worker, layer), or nullptr
+    float* bn_out;               // bucket norms of this message for this (worker, layer)
+    int q;
+    double energy;               // this lane's share of the sum of squared bucket norms
+    uint32_t flags;              // bit 0: a bucket held NaN or Inf, bit 1: a bucket with a nonzero norm
+};
+
+// The L^q norms of the 8 rows (buckets) of the block in this lane's ring slots, all at once.  Every lane forms its
+// fp64 partial of each row; a butterfly that halves the set of rows a lane carries at each of its first three steps
+// leaves the total of row (lane >> 2) in every lane, so the root, the rounding to fp32, the checks and the
+// reciprocal run once per block, for all 8 rows in parallel.  Returns this lane's row's norm (0 for a bucket that is
+// all zero, below the smallest normal float, or non-finite: then `bad`) and its fp32 reciprocal (or 0).
+template <bool kMax>
+__device__ __forceinline__ double pair_op(double x, double y) { return kMax ? fmax(x, y) : x + y; }
+
+template <bool kMax>
+__device__ __forceinline__ double rows_butterfly(double (&part)[8], int lane)
+{
+    const bool h16 = lane & 16, h8 = lane & 8, h4 = lane & 4;
+    double s[4], t[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        s[i] = pair_op<kMax>(h16 ? part[4 + i] : part[i], __shfl_xor_sync(0xffffffffu, h16 ? part[i] : part[4 + i], 16));
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        t[i] = pair_op<kMax>(h8 ? s[2 + i] : s[i], __shfl_xor_sync(0xffffffffu, h8 ? s[i] : s[2 + i], 8));
+    double tot = pair_op<kMax>(h4 ? t[1] : t[0], __shfl_xor_sync(0xffffffffu, h4 ? t[0] : t[1], 4));
+    tot = pair_op<kMax>(tot, __shfl_xor_sync(0xffffffffu, tot, 2));
+    tot = pair_op<kMax>(tot, __shfl_xor_sync(0xffffffffu, tot, 1));
+    return tot;
+}
+
+// mode 0: max |v|   1: sum |v|   2: sum v^2   3: sum |v|^q (integer q >= 3)
+template <int kMode>
+__device__ __forceinline__ void row_partials(const float4* ring_ptr, int q, uint32_t badbits, double (&part)[8])
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float4 v = ring_ptr[32 * j];
+        const float a[4] = {fabsf(v.x), fabsf(v.y), fabsf(v.z), fabsf(v.w)};
+        double acc = 0.0;
+        if (kMode == 0) {
+            acc = (double)fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const double x = (double)a[e];
+                if (kMode == 1)      acc += x;
+                else if (kMode == 2) acc = fma(x, x, acc);
+                else { double pw = x; for (int r = 1; r < q; ++r) pw = __dmul_rn(pw, x); acc += pw; }
+            }
+        }
+        part[j] = ((badbits >> j) & 1u) ? 0.0 : acc;     // a row with NaN or Inf is zeroed whatever it sums to
+    }
+}
+
+__device__ __forceinline__ void bucket_norms8(const float4* ring_ptr, int q, int lane, float& norm, float& rnorm,
+                                              bool& bad)
+{
+    // per row, the largest |v| of this lane as an integer pattern: >= 0x7f800000 means NaN or Inf, 0 means all zero
+    uint32_t badbits = 0, nzbits = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint4 w = *reinterpret_cast<const uint4*>(ring_ptr + 32 * j);
+        const uint32_t mb = max(max(w.x & 0x7fffffffu, w.y & 0x7fffffffu), max(w.z & 0x7fffffffu, w.w & 0x7fffffffu));
+        badbits |= ((mb + 0x00800000u) >> 31) << j;      // mb <= 0x7fffffff: the sum reaches bit 31 iff mb >= 0x7f800000
+        nzbits |= ((mb + 0x7fffffffu) >> 31) << j;       // ... iff mb >= 1
+    }
+    badbits = __reduce_or_sync(0xffffffffu, badbits);
+    nzbits = __reduce_or_sync(0xffffffffu, nzbits);
+    norm = 0.0f; rnorm = 0.0f; bad = false;
+    if ((badbits | nzbits) == 0u) return;                // a block of zeros (untouched embedding rows): nothing to reduce
+    double part[8];
+    double tot;
+    if (q == 0)      { row_partials<0>(ring_ptr, q, badbits, part); tot = rows_butterfly<true>(part, lane); }
+    else if (q == 1) { row_partials<1>(ring_ptr, q, badbits, part); tot = rows_butterfly<false>(part, lane); }
+    else if (q == 2) { row_partials<2>(ring_ptr, q, badbits, part); tot = rows_butterfly<false>(part, lane); }
+    else             { row_partials<3>(ring_ptr, q, badbits, part); tot = rows_butterfly<false>(part, lane); }
+    const int row = lane >> 2;
+    const double n64 = (q == 0 || q == 1) ? tot : (q == 2 ? sqrt(tot) : pow(tot, 1.0 / (double)q));
+    const float n = (float)n64;
+    bad = ((badbits >> row) & 1u) || !(fabs(n64) <= 1.7976931348623157e308) || !(fabsf(n) <= 3.402823466e38f);
+    const bool live = !bad && ((nzbits >> row) & 1u) && n >= 1.17549435e-38f;
+    norm = live ? n : 0.0f;
+    rnorm = live ? __fdiv_rn(1.0f, n) : 0.0f;
+}
+
 // One block of 1024 coordinates from the ring.  `rows` says which of its 8 rows hold anything but
 // zeros (only those were fetched); `next` is this lane's first float4 of the block whose rows
 // replace the consumed ones (nullptr: nothing to fetch) and `next_rows` its row mask; `prev_rows`
 // says which rows may be nonzero in the previous message.  Returns this lane's statistic term.
-template <int B, bool kFast, bool kHist>
+// In bucket scope the value tables hold the plain signed levels and every row brings its own norm.
+template <int B, bool kFast, bool kHist, bool kBucket>
 __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const WarpCtx& c,
                                                  int64_t blk, uint32_t rows, uint32_t prev_rows,
                                                  const float* __restrict__ next, uint32_t next_rows,
                                                  uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
-                                                 QuantSmem& sm)
+                                                 QuantSmem& sm, BucketCtx& bk, float prev_norm8)
 {
+    // prev_norm8 (bucket scope): lanes 0..7 hold the previous message's norms of rows 0..7 of this block
     constexpr int n = 1 << B, C = B + 1;
     const int lane = c.lane;
-    const float r = c.r;
+    float r = c.r;
+    float my_norm = 0.0f, my_rnorm = 0.0f;       // bucket scope: norm and reciprocal of row (lane >> 2)
+    if (kBucket) {
+        bool bad;
+        cp_async_wait<0>();                      // all 8 rows of the block have landed
+        bucket_norms8(c.ring_ptr, bk.q, lane, my_norm, my_rnorm, bad);
+        if ((lane & 3) == 0) bk.energy = fma((double)my_norm, (double)my_norm, bk.energy);
+        bk.flags |= (bad ? 1u : 0u) | (my_norm > 0.0f ? 2u : 0u);
+        if (prev_rows == 0u && !__any_sync(0xffffffffu, my_norm > 0.0f)) {
+            // every bucket of the block is zeroed and the previous message is zero here too: zero words, zero
+            // norms, nothing for the statistic; the ring takes the next block's rows at once
+#pragma unroll
+            for (int j = 0; j < kRingRows; ++j) {
+                if (next && ((next_rows >> j) & 1u)) cp_async16(c.ring + 512u * j, next + 128 * j, 16);
+                cp_async_commit();
+            }
+            const int64_t woff = blk * (int64_t)C * 32 + lane;
+#pragma unroll
+            for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, 0u);
+            if ((lane & 3) == 0) bk.bn_out[blk * 8 + (lane >> 2)] = 0.0f;
+            return 0.0;
+        }
+    }
     uint32_t cw[C];
 #pragma unroll
     for (int w = 0; w < C; ++w) cw[w] = 0u;
@@ -190,7 +305,14 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
 
 #pragma unroll
     for (int j = 0; j < kRingRows; ++j) {
-        const bool live = (rows >> j) & 1u;              // the same for the whole warp
+        bool live = (rows >> j) & 1u;                    // the same for the whole warp
+        float nrow = 0.0f, pn = 0.0f;                    // bucket scope: this row's norm now and in the previous message
+        if (kBucket) {
+            nrow = __shfl_sync(0xffffffffu, my_norm, 4 * j);
+            r = __shfl_sync(0xffffffffu, my_rnorm, 4 * j);
+            live = nrow > 0.0f;                          // a zeroed bucket sends zeros and draws nothing
+            pn = __shfl_sync(0xffffffffu, prev_norm8, j);
+        }
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live) {
             cp_async_wait<kRingRows - 1>();
@@ -242,15 +364,17 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 }
 
                 // step-size statistic: fp32 difference of the two decoded values, squared in fp64
-                const float cur = *reinterpret_cast<const float*>(tcur_b + sym4);
-                const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, pp));
+                float cur = *reinterpret_cast<const float*>(tcur_b + sym4);
+                float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, pp));
+                if (kBucket) { cur = __fmul_rn(cur, nrow); prv = __fmul_rn(prv, pn); }
                 const double dd = (double)__fsub_rn(cur, prv);
                 stat = fma(dd, dd, stat);
             }
         } else if ((prev_rows >> j) & 1u) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, 4 * j + e));
+                float prv = *reinterpret_cast<const float*>(tprev_b + symbol4_at<C>(pw, 4 * j + e));
+                if (kBucket) prv = __fmul_rn(prv, pn);
                 const double dd = (double)prv;
                 stat = fma(dd, dd, stat);
             }
@@ -261,6 +385,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
     const int64_t woff = blk * (int64_t)C * 32 + lane;
 #pragma unroll
     for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, cw[w]);
+    if (kBucket && (lane & 3) == 0) bk.bn_out[blk * 8 + (lane >> 2)] = my_norm;
     return stat;
 }
 
@@ -292,10 +417,10 @@ __device__ __forceinline__ double zeroed_tile(const Tile& tile, int lane, uint32
 // A warp's share of a tile: blocks warp, warp + 8, ...  A block whose rows are all zero in this input and
 // in the input behind the previous message is an all-zero piece of message that adds nothing to the
 // statistic: its words are stored and nothing is read.
-template <int B, bool kFast, bool kHist>
+template <int B, bool kFast, bool kHist, bool kBucket>
 __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const WarpCtx& c, const Tile& tile,
                                                 uint32_t* __restrict__ out,
-                                                const uint32_t* __restrict__ prev, QuantSmem& sm)
+                                                const uint32_t* __restrict__ prev, QuantSmem& sm, BucketCtx& bk)
 {
     constexpr int C = B + 1;
     const int warp = threadIdx.x >> 5;
@@ -323,9 +448,16 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
                 issue_ragged_block(c, blk);
             }
         }
+        float prev_norm8 = 0.0f;
+        uint32_t pmask = prows;
+        if (kBucket && prev) {
+            // the previous message's norms tell which of its rows are all zero: those add nothing to the statistic
+            if (c.lane < 8) prev_norm8 = __ldg(bk.prev_bn + blk * 8 + c.lane);
+            pmask = __ballot_sync(0xffffffffu, prev_norm8 != 0.0f) & 0xffu;
+        }
         uint32_t pw[C];
 #pragma unroll
-        for (int w = 0; w < C; ++w) pw[w] = (prev && prows) ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
+        for (int w = 0; w < C; ++w) pw[w] = (prev && pmask) ? __ldcs(prev + blk * (int64_t)C * 32 + c.lane + w * 32) : 0u;
         // the next block of this warp that has anything in it: its rows replace the consumed ones
         int nb = b + kQWarps;
         while (nb < tile.nblocks && (sm.rows_cur[nb] | sm.rows_prev[nb]) == 0u) {
@@ -338,7 +470,7 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
         const int64_t nblk = tile.block0 + nb;
         const uint32_t next_rows = has_next ? sm.rows_cur[nb] : 0u;
         const float* next = (has_next && nblk < nfull) ? c.g + nblk * kBlockCoords + 4 * c.lane : nullptr;
-        stat += quantize_block<B, kFast, kHist>(pc, c, blk, rows, prows, next, next_rows, out, pw, sm);
+        stat += quantize_block<B, kFast, kHist, kBucket>(pc, c, blk, rows, pmask, next, next_rows, out, pw, sm, bk, prev_norm8);
         primed = has_next;
         if (has_next && nblk >= nfull) issue_ragged_block(c, nblk);   // the layer's last, partial block
         b = nb - kQWarps;                                             // the loop's increment lands on nb
@@ -347,10 +479,10 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
     return stat;
 }
 
-template <bool kHist>
+template <bool kHist, bool kBucket>
 __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     PlanDev p, const float* __restrict__ grads, uint32_t step, uint32_t* __restrict__ packed,
-    const float* __restrict__ norms, uint32_t* __restrict__ hist,
+    const float* __restrict__ norms, float* __restrict__ bucket_norms, uint32_t* __restrict__ hist,
     const uint32_t* __restrict__ prev_packed, const float* __restrict__ prev_norms,
     const float* __restrict__ levels_cur, const float* __restrict__ levels_prev, SearchTables st)
 {
@@ -362,8 +494,9 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     const int k = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t kl = (int64_t)k * p.num_layers + layer;
-    const float ncur = norms[kl];
-    const float nprev = prev_norms ? prev_norms[kl] : 0.0f;
+    // bucket scope: the tables hold the plain levels (norm 1) and each row multiplies by its own norm
+    const float ncur = kBucket ? 1.0f : norms[kl];
+    const float nprev = kBucket ? 1.0f : (prev_norms ? prev_norms[kl] : 0.0f);
     const bool fast = st.fast[layer] != 0;
     const int n = L.nlevels;
 
@@ -385,8 +518,9 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
         // with a histogram every coordinate counts, zero or not, so every row is fetched; a previous
         // message whose masks are unknown is taken as nonzero everywhere
         const int64_t mb = (int64_t)k * p.total_blocks + L.block_off + tile.block0 + threadIdx.x;
-        sm.rows_cur[threadIdx.x] = kHist ? (uint8_t)0xff : p.row_mask[mb];
-        sm.rows_prev[threadIdx.x] = !prev_packed ? (uint8_t)0 : (p.row_mask_prev ? p.row_mask_prev[mb] : (uint8_t)0xff);
+        sm.rows_cur[threadIdx.x] = (kHist || kBucket) ? (uint8_t)0xff : p.row_mask[mb];
+        sm.rows_prev[threadIdx.x] = !prev_packed ? (uint8_t)0
+                                    : ((p.row_mask_prev && !kBucket) ? p.row_mask_prev[mb] : (uint8_t)0xff);
     }
     __syncthreads();
 
@@ -395,9 +529,15 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     c.size = L.size;
     c.ring_ptr = ring_mem + (warp * kRingRows) * 32 + lane;
     c.ring = (uint32_t)__cvta_generic_to_shared(c.ring_ptr);
-    c.r = p.rnorm[kl];
+    c.r = kBucket ? 1.0f : p.rnorm[kl];
     c.lane = lane;
     const bool zeroed = c.r == 0.0f;
+    BucketCtx bk{nullptr, nullptr, p.q, 0.0, 0u};
+    if (kBucket) {
+        const int64_t bo = (int64_t)k * p.total_blocks * 8 + L.block_off * 8;
+        bk.prev_bn = prev_norms ? prev_norms + bo : nullptr;
+        bk.bn_out = bucket_norms + bo;
+    }
     const PhiloxConsts pc = philox_fold((uint32_t)layer, (uint32_t)k, step, p.seed_lo, p.seed_hi);
     uint32_t* out = packed + (int64_t)k * p.packed_words + L.word_off;
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
@@ -406,14 +546,23 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     switch (zeroed ? -L.bits : L.bits * 2 + (fast ? 1 : 0)) {
 #define LQ_CASE(BB)                                                                              \
     case -BB:        stat = zeroed_tile<BB>(tile, lane, out, prev, sm); break;                   \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(pc, c, tile, out, prev, sm); break;  \
-    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(pc, c, tile, out, prev, sm); break;
+    case 2 * BB:     stat = quantize_tile<BB, false, kHist, kBucket>(pc, c, tile, out, prev, sm, bk); break;  \
+    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist, kBucket>(pc, c, tile, out, prev, sm, bk); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
     }
     const double total = block_reduce<false>(stat, sm.scratch);
     if (threadIdx.x == 0) p.stat_partial[(int64_t)k * p.num_tiles + blockIdx.x] = total;
+    if (kBucket) {
+        const double energy = block_reduce<false>(bk.energy, sm.scratch);
+        const int any_bad = __syncthreads_or((int)(bk.flags & 1u));
+        const int any_live = __syncthreads_or((int)(bk.flags & 2u));
+        if (threadIdx.x == 0) {
+            p.energy_partial[(int64_t)k * p.num_tiles + blockIdx.x] = energy;
+            p.flag_partial[(int64_t)k * p.num_tiles + blockIdx.x] = (any_bad ? 1u : 0u) | (any_live ? 2u : 0u);
+        }
+    }
 
     if (kHist) {
         __syncthreads();
@@ -434,6 +583,34 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
     for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) acc += part[i];
     const double total = block_reduce<false>(acc, scratch);
     if (threadIdx.x == 0) p.sq_diff[(int64_t)k * p.num_layers + m] = total;
+}
+
+// Bucket scope: per (layer, worker), in tile order: the statistic, the layer's energy (its weight in the level fit,
+// as the square root of the summed squared bucket norms) and its flags: LQ_STATUS_NONFINITE if a bucket was
+// zeroed because it held NaN or Inf, else LQ_STATUS_ZERO_NORM if no bucket has a nonzero norm.
+__global__ void __launch_bounds__(128) bucket_finalize_kernel(PlanDev p)
+{
+    __shared__ double scratch[4];
+    const int m = blockIdx.x, k = blockIdx.y;
+    const LayerDesc L = p.layers[m];
+    const int64_t o = (int64_t)k * p.num_tiles + L.first_tile;
+    double acc = 0.0, en = 0.0;
+    uint32_t fl = 0;
+    for (int i = threadIdx.x; i < L.ntiles; i += blockDim.x) {
+        acc += p.stat_partial[o + i];
+        en += p.energy_partial[o + i];
+        fl |= p.flag_partial[o + i];
+    }
+    const double total = block_reduce<false>(acc, scratch);
+    const double energy = block_reduce<false>(en, scratch);
+    const int any_bad = __syncthreads_or((int)(fl & 1u));
+    const int any_live = __syncthreads_or((int)(fl & 2u));
+    if (threadIdx.x == 0) {
+        const int64_t kl = (int64_t)k * p.num_layers + m;
+        p.sq_diff[kl] = total;
+        p.layer_weight[kl] = (float)sqrt(energy);
+        p.status[kl] = any_bad ? LQ_STATUS_NONFINITE : (any_live ? 0u : LQ_STATUS_ZERO_NORM);
+    }
 }
 
 // One CTA per layer: derives the encode-side tables from the layer's levels.
@@ -487,11 +664,33 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
     if (p.num_tiles == 0) return cudaSuccess;
     const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
     if (hist)
-        quantize_pack_kernel<true><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist,
-                                                                         prev_packed, prev_norms, levels_cur, levels_prev, t);
+        quantize_pack_kernel<true, false><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, nullptr, hist,
+                                                                                prev_packed, prev_norms, levels_cur, levels_prev, t);
     else
-        quantize_pack_kernel<false><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, hist,
-                                                                          prev_packed, prev_norms, levels_cur, levels_prev, t);
+        quantize_pack_kernel<false, false><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, nullptr, hist,
+                                                                                 prev_packed, prev_norms, levels_cur, levels_prev, t);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
+                                     float* bucket_norms, uint32_t* hist, const uint32_t* prev_packed,
+                                     const float* prev_norms, const float* levels_cur,
+                                     const float* levels_prev, SearchTables t, cudaStream_t s)
+{
+    if (p.num_tiles == 0) return cudaSuccess;
+    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
+    if (hist)
+        quantize_pack_kernel<true, true><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, nullptr, bucket_norms, hist,
+                                                                               prev_packed, prev_norms, levels_cur, levels_prev, t);
+    else
+        quantize_pack_kernel<false, true><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, nullptr, bucket_norms, hist,
+                                                                                prev_packed, prev_norms, levels_cur, levels_prev, t);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bucket_finalize(const PlanDev& p, cudaStream_t s)
+{
+    bucket_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p);
     return cudaGetLastError();
 }
 

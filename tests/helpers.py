@@ -55,3 +55,19 @@ def compare_messages(orc, plan, packed_gpu: torch.Tensor, ref: dict):
             if not diff.any():
                 stray_words += int((got != want).sum())
     return bad_coords, stray_words
+
+
+def bucket_norms_by_layer(plan, nm: torch.Tensor):
+    """Bucket scope: the [K][8 * blocks] norms buffer -> per layer an array [K][ceil(d / 128)], plus the largest
+    absolute value found in the slots of rows past the layers' ends (must be 0)."""
+    a = nm.detach().cpu().numpy()
+    out, stray, block_off = [], 0.0, 0
+    for d in plan.layer_sizes:
+        nblocks = (d + 1023) // 1024
+        nb = (d + 127) // 128
+        seg = a[:, 8 * block_off: 8 * (block_off + nblocks)]
+        out.append(seg[:, :nb].copy())
+        if seg[:, nb:].size:
+            stray = max(stray, float(np.abs(seg[:, nb:]).max()))
+        block_off += nblocks
+    return out, stray
