@@ -219,6 +219,14 @@ def run_gpu(args) -> None:
     grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, dev)
     packed = [plan.empty_packed(dev), plan.empty_packed(dev)]
     norms = [plan.empty_norms(dev), plan.empty_norms(dev)]
+    ex = None
+    if args.exchange:
+        # the K workers are shared out over the ranks; messages travel by all-gather (strong scaling)
+        from paper_2505_14371_b200.exchange import ExchangeStep
+        ex = ExchangeStep(plan, rank, world, device=dev)
+        grads = grads[ex.first: ex.first + ex.count].contiguous()
+        del packed, norms
+    share = 1.0 / world if args.exchange else 1.0     # this rank's part of the job's 4 K D input bytes
     g = torch.Generator(device=dev).manual_seed(W.SEED_BASE + 99)
     X1 = torch.randn(plan.padded_elems, generator=g, device=dev)
     Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
@@ -229,6 +237,9 @@ def run_gpu(args) -> None:
     def step():
         state["t"] += 1
         t = state["t"]
+        if ex is not None:
+            ex.step(grads, t, X1, Y, Xh)
+            return
         c, p = t % 2, (t + 1) % 2
         plan.lq_quantize_pack(grads, t, packed[c], norms[c],
                               prev_packed=None if t == 1 else packed[p],
@@ -238,9 +249,13 @@ def run_gpu(args) -> None:
     # adaptive levels: one histogram + fit before the steady state (Algorithm 1 lines 2-7)
     hist = plan.zero_hist(dev)
     state["t"] += 1
-    plan.lq_quantize_pack(grads, 1, packed[1], norms[1], hist=hist)
-    plan.lq_fit_levels(hist, norms[1], K)
-    plan.qoda_step(packed[1], norms[1], X1, Y, Xh)
+    if ex is not None:
+        ex.step(grads, 1, X1, Y, Xh, hist=hist)
+        ex.fit_levels(hist)
+    else:
+        plan.lq_quantize_pack(grads, 1, packed[1], norms[1], hist=hist)
+        plan.lq_fit_levels(hist, norms[1], K)
+        plan.qoda_step(packed[1], norms[1], X1, Y, Xh)
     del hist
     for _ in range(max(args.warmup, 3)):
         step()
@@ -290,7 +305,7 @@ def run_gpu(args) -> None:
         e1.record()
         barrier()
         e2e_ms = aggregate_over_ranks(e0.elapsed_time(e1) / e2e_steps, world, dev)
-        e2e = {"value": whole_job_value(4.0 * K * D / 1e9, world, e2e_ms), "unit": "GB/s",
+        e2e = {"value": whole_job_value(4.0 * K * D * share / 1e9, world, e2e_ms), "unit": "GB/s",
                "h2d_bytes_per_step": host_grads.numel() * 4, "d2h_bytes_per_step": host_out.numel() * 4,
                "ms_per_step": e2e_ms}
         del host_grads, host_out
@@ -316,6 +331,11 @@ def run_gpu(args) -> None:
         cb = c + 4.0 / 128.0
         alg = {"quantize_pack": (4.0 + 2 * cb) * K * D, "decode": (K * cb + 16.0) * D}
         qp_alg = alg["quantize_pack"]
+    if args.exchange:                         # a rank encodes only its share of the workers (and decodes all of them)
+        for name in ("norm_partial", "quantize_pack"):
+            if name in alg:
+                alg[name] *= share
+        qp_alg *= share
     kern = {}
     for name, (tot, cnt) in prof.items():
         if cnt:
@@ -349,14 +369,15 @@ def run_gpu(args) -> None:
 
     cpu = time_oracle(3, 0) if world == 1 and not args.no_cpu_baseline else None
     launches = int(sum(cnt for _, cnt in prof.values()))
-    line = {"metric": METRIC, "value": whole_job_value(4.0 * K * D / 1e9, world, ms), "unit": "GB/s",
+    line = {"metric": METRIC, "value": whole_job_value(4.0 * K * D * share / 1e9, world, ms), "unit": "GB/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "higher_is_better": True, "scaling": "strong" if args.exchange else "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": f"{w.name}_shaped", "coords": D, "layers": w.num_layers, "num_workers": K,
                        "bits": w.bits, "q": w.q, "norm_scope": args.norm_scope, "levels": "adaptive (fitted once before timing)",
                        "l2": "inputs (%.2f GB) exceed L2" % (4.0 * K * D / 1e9),
-                       "multi_gpu": "replicas only"},
+                       "multi_gpu": "K workers shared out over the ranks, messages by all-gather" if args.exchange
+                                    else "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "calls": calls}
     if cpu:
         line["cpu_baseline"] = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
@@ -445,6 +466,9 @@ def main() -> None:
     ap.add_argument("--workload", default="transformer_xl")
     ap.add_argument("--norm-scope", default="layer", choices=["layer", "global", "bucket"],
                     help="layer: one norm per layer (the headline configuration); bucket: one per 128 coordinates")
+    ap.add_argument("--exchange", action="store_true",
+                    help="share the K workers out over the ranks and exchange the messages by all-gather (default: "
+                         "every rank runs the whole K-worker job on its own data)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, widths, workers, norms")
     ap.add_argument("--sweep-quick", action="store_true")

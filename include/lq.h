@@ -103,6 +103,24 @@ int lq_plan_layer_info(const lq_plan* plan, int32_t layer, int64_t* elem_off, in
 #define LQ_NORM_BUCKET    2
 #define LQ_BUCKET         128
 int lq_set_norm_scope(lq_plan* plan, int32_t scope);
+/* Worker range (several processes sharing one job: Algorithm 1 has every node encode its own dual vector and
+ * broadcast it).  After lq_set_worker_range(plan, first, count) the encode-side calls - lq_layer_norms and
+ * lq_quantize_pack - handle only workers first .. first + count - 1: `grads` is [count][D_pad] (row 0 = worker
+ * `first`), while packed, norms, hist, prev_packed and prev_norms keep their full [K] shapes and only the rows of
+ * the range are read or written; the random numbers are those of the workers' global indices, so K processes of
+ * one worker each emit the same messages as one process of K workers.  The caller then brings the other workers'
+ * rows of packed and norms in (an all-gather), and their per-(worker, layer) side data - the step-size statistic
+ * that qoda_step consumes, the bucket scope's fit weights, the flags - with the two calls below, before
+ * lq_decode_aggregate / qoda_step / lq_fit_levels, which always cover all K workers.  Default range: (0, K).
+ * LQ_EINVAL if the range does not lie inside [0, K). */
+int lq_set_worker_range(lq_plan* plan, int32_t first_worker, int32_t count);
+/* Copies the plan's per-(worker, layer) side data to / from DEVICE arrays of shape [K][L] on `stream`
+ * (sq_diff fp64, 8-byte aligned; layer_weight fp32; flags u32; any pointer may be NULL = skip).  Export after
+ * lq_quantize_pack, exchange the rows, import before qoda_step. */
+int lq_side_data_export(const lq_plan* plan, double* sq_diff, float* layer_weight, uint32_t* flags, void* stream);
+int lq_side_data_import(lq_plan* plan, const double* sq_diff, const float* layer_weight, const uint32_t* flags,
+                        void* stream);
+
 /* fp32 values per worker in a norms buffer under the plan's current scope: the number of layers, or in bucket
  * scope 8 x the number of 1024-coordinate blocks of all layers.  Negative error code on failure. */
 int64_t lq_plan_norm_count(const lq_plan* plan);

@@ -22,7 +22,8 @@ STATUS_ZERO_NORM = 1
 STATUS_NONFINITE = 2
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
-           "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
+           "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_worker_range", "lq_side_data_export",
+           "lq_side_data_import", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_code_build", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
            "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
@@ -58,6 +59,9 @@ def load_library() -> C.CDLL:
     L.lq_plan_norm_count.argtypes = [vp]
     L.lq_plan_norm_count.restype = i64
     L.lq_layer_weights.argtypes = [vp, vp]
+    L.lq_set_worker_range.argtypes = [vp, i32, i32]
+    L.lq_side_data_export.argtypes = [vp, vp, vp, vp, vp]
+    L.lq_side_data_import.argtypes = [vp, vp, vp, vp, vp]
     L.lq_set_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_get_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
     L.lq_layer_norms.argtypes = [vp, vp, vp, vp]
@@ -172,6 +176,17 @@ class Plan:
         """"layer" (default), "global" (one norm over the worker's whole vector) or "bucket" (one norm per 128
         consecutive coordinates of a layer; norms buffers then have lq_plan_norm_count() values per worker)."""
         _check(load_library().lq_set_norm_scope(self._h, {"layer": 0, "global": 1, "bucket": 2}[scope]))
+
+    def lq_set_worker_range(self, first_worker: int, count: int) -> None:
+        _check(load_library().lq_set_worker_range(self._h, int(first_worker), int(count)))
+
+    def lq_side_data_export(self, sq_diff=None, layer_weight=None, flags=None) -> None:
+        _check(load_library().lq_side_data_export(self._h, _ptr(sq_diff, torch.float64), _ptr(layer_weight, torch.float32),
+                                                  _ptr(flags, torch.int32), _stream()))
+
+    def lq_side_data_import(self, sq_diff=None, layer_weight=None, flags=None) -> None:
+        _check(load_library().lq_side_data_import(self._h, _ptr(sq_diff, torch.float64), _ptr(layer_weight, torch.float32),
+                                                  _ptr(flags, torch.int32), _stream()))
 
     def lq_plan_norm_count(self) -> int:
         n = int(load_library().lq_plan_norm_count(self._h))

@@ -217,6 +217,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     p->seed = seed;
     PlanDev& d = p->dev;
     d.num_layers = num_layers; d.num_tiles = (int32_t)ntiles; d.num_workers = num_workers; d.q = q;
+    d.worker0 = 0; d.worker_count = num_workers;
     d.sub_tiles = tile_blocks / kSubBlocks;
     d.sub_shift = 0;
     while ((1 << d.sub_shift) < d.sub_tiles) ++d.sub_shift;
@@ -530,6 +531,41 @@ int lq_set_norm_scope(lq_plan* plan, int32_t scope)
         return fail(LQ_ESTATE, "the bucket scope can only be entered or left before the first lq_quantize_pack");
     plan->dev.global_norm = scope == LQ_NORM_GLOBAL ? 1 : 0;
     plan->dev.bucket_norm = bucket;
+    return LQ_OK;
+}
+
+int lq_set_worker_range(lq_plan* plan, int32_t first_worker, int32_t count)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    if (first_worker < 0 || count < 1 || first_worker > plan->dev.num_workers - count)
+        return fail(LQ_EINVAL, "worker range [%d, %d) is not inside [0, %d)", first_worker, first_worker + count,
+                    plan->dev.num_workers);
+    plan->dev.worker0 = first_worker;
+    plan->dev.worker_count = count;
+    return LQ_OK;
+}
+
+int lq_side_data_export(const lq_plan* plan, double* sq_diff, float* layer_weight, uint32_t* flags, void* stream)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    LQ_ALIGNED(sq_diff, 8); LQ_ALIGNED(layer_weight, 4); LQ_ALIGNED(flags, 4);
+    const size_t KL = (size_t)plan->dev.num_workers * (size_t)plan->dev.num_layers;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (sq_diff) LQ_CUDA(cudaMemcpyAsync(sq_diff, plan->dev.sq_diff, KL * sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (layer_weight) LQ_CUDA(cudaMemcpyAsync(layer_weight, plan->dev.layer_weight, KL * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    if (flags) LQ_CUDA(cudaMemcpyAsync(flags, plan->dev.status, KL * sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
+    return LQ_OK;
+}
+
+int lq_side_data_import(lq_plan* plan, const double* sq_diff, const float* layer_weight, const uint32_t* flags, void* stream)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    LQ_ALIGNED(sq_diff, 8); LQ_ALIGNED(layer_weight, 4); LQ_ALIGNED(flags, 4);
+    const size_t KL = (size_t)plan->dev.num_workers * (size_t)plan->dev.num_layers;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (sq_diff) LQ_CUDA(cudaMemcpyAsync(plan->dev.sq_diff, sq_diff, KL * sizeof(double), cudaMemcpyDeviceToDevice, s));
+    if (layer_weight) LQ_CUDA(cudaMemcpyAsync(plan->dev.layer_weight, layer_weight, KL * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    if (flags) LQ_CUDA(cudaMemcpyAsync(plan->dev.status, flags, KL * sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
     return LQ_OK;
 }
 

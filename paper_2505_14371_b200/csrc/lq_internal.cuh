@@ -64,6 +64,8 @@ struct PlanDev {
     int32_t sub_shift;    // log2(sub_tiles)
     int32_t global_norm;  // 1: one norm per worker over all layers (Section 3.1), 0: one per layer
     int32_t bucket_norm;  // 1: one norm per bucket of 128 consecutive coordinates of a layer (Section 7.1)
+    int32_t worker0;      // the encode-side kernels cover workers worker0 .. worker0 + worker_count - 1 (grid.y =
+    int32_t worker_count; // worker_count); `grads` holds only those rows, every other buffer all K rows
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;

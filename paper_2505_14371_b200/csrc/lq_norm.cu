@@ -38,9 +38,9 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
     const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;          // this CTA's blocks of the tile
     const int sub1 = min(sub0 + kSubBlocks, tile.nblocks);
     const LayerDesc L = p.layers[tile.layer];
-    const int k = blockIdx.y;
+    const int k = blockIdx.y + p.worker0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float* __restrict__ g = grads + (int64_t)k * p.padded_elems + L.elem_off;
+    const float* __restrict__ g = grads + (int64_t)blockIdx.y * p.padded_elems + L.elem_off;
 
     double acc = 0.0;
     uint32_t maxbits = 0;
@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const
 __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __restrict__ norms)
 {
     __shared__ double scratch[4];
-    const int m = blockIdx.x, k = blockIdx.y;
+    const int m = blockIdx.x, k = blockIdx.y + p.worker0;
     const LayerDesc L = p.layers[m];
     const double* part = p.norm_partial + ((int64_t)k * p.num_tiles + L.first_tile) * p.sub_tiles;
     double acc = 0.0;
@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(128) norm_global_kernel(PlanDev p, float* __re
     __shared__ double scratch[4];
     __shared__ float n_s;
     __shared__ uint32_t st_s;
-    const int k = blockIdx.x;
+    const int k = blockIdx.x + p.worker0;
     const double* tot = p.layer_total + (int64_t)k * p.num_layers;
     double acc = 0.0;
     int bad = 0;
@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(128) norm_global_kernel(PlanDev p, float* __re
 cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write_mask, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
-    const dim3 grid((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.num_workers);
+    const dim3 grid((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.worker_count);
     if (p.q == 0)      norm_partial_kernel<0><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
     else if (p.q == 1) norm_partial_kernel<1><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
     else if (p.q == 2) norm_partial_kernel<2><<<grid, kThreads, 0, s>>>(p, grads, write_mask);
@@ -193,8 +193,8 @@ cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write
 
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s)
 {
-    norm_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p, norms);
-    if (p.global_norm) norm_global_kernel<<<(unsigned)p.num_workers, 128, 0, s>>>(p, norms);
+    norm_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.worker_count), 128, 0, s>>>(p, norms);
+    if (p.global_norm) norm_global_kernel<<<(unsigned)p.worker_count, 128, 0, s>>>(p, norms);
     return cudaGetLastError();
 }
 

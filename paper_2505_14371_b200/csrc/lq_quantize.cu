@@ -491,7 +491,7 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     const Tile tile = p.tiles[blockIdx.x];
     const int layer = tile.layer;
     const LayerDesc L = p.layers[layer];
-    const int k = blockIdx.y;
+    const int k = blockIdx.y + p.worker0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t kl = (int64_t)k * p.num_layers + layer;
     // bucket scope: the tables hold the plain levels (norm 1) and each row multiplies by its own norm
@@ -525,7 +525,7 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     __syncthreads();
 
     WarpCtx c;
-    c.g = grads + (int64_t)k * p.padded_elems + L.elem_off;
+    c.g = grads + (int64_t)blockIdx.y * p.padded_elems + L.elem_off;
     c.size = L.size;
     c.ring_ptr = ring_mem + (warp * kRingRows) * 32 + lane;
     c.ring = (uint32_t)__cvta_generic_to_shared(c.ring_ptr);
@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
 __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 {
     __shared__ double scratch[4];
-    const int m = blockIdx.x, k = blockIdx.y;
+    const int m = blockIdx.x, k = blockIdx.y + p.worker0;
     const LayerDesc L = p.layers[m];
     const double* part = p.stat_partial + (int64_t)k * p.num_tiles + L.first_tile;
     double acc = 0.0;
@@ -591,7 +591,7 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 __global__ void __launch_bounds__(128) bucket_finalize_kernel(PlanDev p)
 {
     __shared__ double scratch[4];
-    const int m = blockIdx.x, k = blockIdx.y;
+    const int m = blockIdx.x, k = blockIdx.y + p.worker0;
     const LayerDesc L = p.layers[m];
     const int64_t o = (int64_t)k * p.num_tiles + L.first_tile;
     double acc = 0.0, en = 0.0;
@@ -662,7 +662,7 @@ cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step,
                             const float* levels_prev, SearchTables t, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
-    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
+    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.worker_count);
     if (hist)
         quantize_pack_kernel<true, false><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, norms, nullptr, hist,
                                                                                 prev_packed, prev_norms, levels_cur, levels_prev, t);
@@ -678,7 +678,7 @@ cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint3
                                      const float* levels_prev, SearchTables t, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
-    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.num_workers);
+    const dim3 grid((unsigned)p.num_tiles, (unsigned)p.worker_count);
     if (hist)
         quantize_pack_kernel<true, true><<<grid, kQThreads, kRingBytes, s>>>(p, grads, step, packed, nullptr, bucket_norms, hist,
                                                                                prev_packed, prev_norms, levels_cur, levels_prev, t);
@@ -690,13 +690,13 @@ cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint3
 
 cudaError_t launch_bucket_finalize(const PlanDev& p, cudaStream_t s)
 {
-    bucket_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p);
+    bucket_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.worker_count), 128, 0, s>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s)
 {
-    stat_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.num_workers), 128, 0, s>>>(p);
+    stat_finalize_kernel<<<dim3((unsigned)p.num_layers, (unsigned)p.worker_count), 128, 0, s>>>(p);
     return cudaGetLastError();
 }
 

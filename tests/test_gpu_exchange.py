@@ -1,0 +1,42 @@
+"""The exchange path (one process per worker range, messages by all-gather) against one process holding all K
+workers: bit-identical messages, iterates and step sizes.  The two ranks run as child processes on the same GPU
+with the gloo backend: their kernels never wait on one another (the collectives run on the host)."""
+import os
+import socket
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def _free_port() -> str:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return str(s.getsockname()[1])
+
+
+@pytest.mark.parametrize("scope", ["layer", "bucket"])
+def test_two_ranks_equal_one_process(tmp_path, scope):
+    sys.path.insert(0, HERE)
+    import exchange_rank
+    want = exchange_rank.run(0, 1, scope, False)                  # all K workers in this process
+    port = _free_port()
+    procs = [subprocess.Popen([sys.executable, os.path.join(HERE, "exchange_rank.py"), str(r), "2", port,
+                               str(tmp_path), scope], stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+             for r in range(2)]
+    outs = []
+    for p in procs:
+        try:
+            outs.append(p.communicate(timeout=300)[0])
+        except subprocess.TimeoutExpired:
+            p.kill()
+            outs.append(p.communicate()[0])
+    assert all(p.returncode == 0 for p in procs), "\n".join(outs)
+    for r in range(2):
+        got = np.load(tmp_path / f"rank{r}.npz")
+        for key in want:
+            assert np.array_equal(got[key], want[key]), (r, key)

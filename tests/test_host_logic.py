@@ -127,3 +127,95 @@ def test_library_code_builder_is_optimal_like_the_oracles(orc):
     assert binding.lq_code_build([0.4, 0.3, 0.2, 0.1]) == [1, 2, 3, 3]
     with pytest.raises(binding.LqError):
         binding.lq_code_build([0.5, -0.1])
+
+
+# ---------------------------------------------------------------------------------------------- exchange plumbing
+class _FakePlan:
+    """Stands in for a Plan on a machine without a GPU: records the call order and lets "encode" write
+    worker-specific values into the rows of its range, so that the all-gather's assembly can be checked."""
+
+    def __init__(self, K, L, W):
+        self.num_workers, self.num_layers, self.W = K, L, W
+        self.calls = []
+
+    def lq_set_worker_range(self, first, count):
+        self.first, self.count = first, count
+
+    def empty_packed(self, device):
+        import torch
+        return torch.empty((self.num_workers, self.W), dtype=torch.int32, device=device)
+
+    def empty_norms(self, device):
+        import torch
+        return torch.empty((self.num_workers, self.num_layers), dtype=torch.float32, device=device)
+
+    def lq_quantize_pack(self, grads, step, packed, norms, hist=None, prev_packed=None, prev_norms=None):
+        self.calls.append(("quantize", step, prev_packed is not None))
+        for i in range(self.count):
+            k = self.first + i
+            packed[k] = 1000 * step + k
+            norms[k] = float(k) + 0.5
+            if hist is not None:
+                hist[k] = k + 1
+        self.step = step
+
+    def lq_side_data_export(self, sq, w, f):
+        for i in range(self.count):
+            k = self.first + i
+            sq[k] = 10.0 * self.step + k; w[k] = k; f[k] = k % 2
+
+    def lq_side_data_import(self, sq, w, f):
+        self.imported = (sq.clone(), w.clone(), f.clone())
+
+    def qoda_step(self, packed, norms, X1, Y, Xhalf, X, gbar):
+        self.calls.append(("qoda_step",))
+        self.seen = (packed.clone(), norms.clone())
+
+
+def _exchange_rank(rank, world, port, out_dir):
+    import json
+    import os
+    import torch
+    import torch.distributed as dist
+    from paper_2505_14371_b200.exchange import ExchangeStep
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    K, L, W = 4, 3, 8
+    plan = _FakePlan(K, L, W)
+    ex = ExchangeStep(plan, rank, world, device="cpu")
+    hist = torch.zeros((K, L, 4), dtype=torch.int32)
+    for t in (1, 2):
+        ex.step(torch.zeros((ex.count, 16)), t, None, None, None, hist=hist if t == 1 else None)
+    packed, norms = plan.seen
+    sq, w, f = plan.imported
+    ok = all(int(packed[k, 0]) == 2000 + k and float(norms[k, 0]) == k + 0.5 and float(sq[k, 0]) == 20.0 + k
+             and float(w[k, 0]) == k and int(f[k, 0]) == k % 2 and int(hist[k, 0, 0]) == k + 1 for k in range(K))
+    with open(os.path.join(out_dir, f"x{rank}.json"), "w") as fh:
+        json.dump({"ok": ok, "calls": plan.calls, "range": [ex.first, ex.count]}, fh)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_exchange_worker_ranges():
+    from paper_2505_14371_b200.exchange import worker_range
+    assert [worker_range(r, 4, 8) for r in range(4)] == [(0, 2), (2, 2), (4, 2), (6, 2)]
+    assert worker_range(0, 1, 8) == (0, 8)
+    with pytest.raises(ValueError):
+        worker_range(0, 3, 8)
+    with pytest.raises(ValueError):
+        worker_range(2, 2, 8)
+
+
+def test_exchange_assembles_all_rows_with_gloo_two_ranks(tmp_path):
+    import json
+    import socket
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_exchange_rank, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    for r in range(2):
+        rec = json.load(open(tmp_path / f"x{r}.json"))
+        assert rec["ok"] and rec["range"] == [2 * r, 2]
+        # the second message is encoded against the first; each encode is followed by one update
+        assert rec["calls"] == [["quantize", 1, False], ["qoda_step"], ["quantize", 2, True], ["qoda_step"]]
