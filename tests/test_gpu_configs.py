@@ -262,6 +262,72 @@ def test_config4_transformer_xl_full_size_sampled(lqm, orc):
     assert abs(eta - 1.0 / math.sqrt(1.0 + S)) <= 1e-6 * eta
 
 
+def test_config4_bucket_scope_full_size_sampled(lqm, orc):
+    """The same workload in bucket scope (`bench.py --norm-scope bucket`): sampled blocks' bucket norms, symbols and
+    aggregate against the oracle applied bucket by bucket; zero buckets carry norm 0 and leave Y alone."""
+    from paper_2505_14371_b200 import workloads as W
+    if torch.cuda.mem_get_info()[0] < 20e9:
+        pytest.skip("needs about 12 GB of free device memory")
+    w = W.transformer_xl_workload()
+    K, Lr = w.num_workers, w.num_layers
+    plan = lqm.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+    plan.lq_set_norm_scope("bucket")
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda")
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    X1 = torch.zeros(plan.padded_elems, device="cuda")
+    Y = torch.empty_like(X1); Xh = torch.empty_like(X1); gbar = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, pk[1], nm[1], hist=hist)
+    plan.lq_fit_levels(hist, nm[1], K)
+    plan.qoda_step(pk[1], nm[1], X1, Y, Xh)
+    del hist
+    Y_before = Y.clone()
+    plan.lq_quantize_pack(grads, 2, pk[0], nm[0], prev_packed=pk[1], prev_norms=nm[1])
+    plan.qoda_step(pk[0], nm[0], X1, Y, Xh, None, gbar)
+    torch.cuda.synchronize()
+    _, flags = plan.lq_get_statistics()
+    assert int(flags.sum()) == 0
+    levels = [np.array(plan.lq_get_levels(m), np.float32) for m in range(Lr)]
+    C = w.bits + 1
+    block_off = np.concatenate([[0], np.cumsum([(d + 1023) // 1024 for d in w.layer_sizes])])
+    rng = np.random.default_rng(11)
+
+    def check_blocks(m, b0, nb):
+        d = w.layer_sizes[m]
+        lo = b0 * 1024; hi = min(d, lo + nb * 1024)
+        e0 = plan.elem_offsets[m]
+        decoded = np.zeros((K, hi - lo), np.float32)
+        for k in range(K):
+            v = grads[k, e0 + lo: e0 + hi].cpu().numpy()
+            got_bn = nm[0][k, 8 * (block_off[m] + b0): 8 * (block_off[m] + b0 + nb)].cpu().numpy()
+            idx = np.zeros(hi - lo, np.uint8); sg = np.zeros(hi - lo, np.uint8)
+            for i in range(0, hi - lo, 128):
+                seg = v[i: i + 128]
+                bn, _ = orc.layer_norm(seg, w.q)
+                assert got_bn[i // 128] == bn, (m, b0, k, i)
+                idx[i: i + 128], sg[i: i + 128], _ = orc.quantize_layer(seg, bn, levels[m], W.PHILOX_SEED, 2, k, m,
+                                                                         first_index=lo + i)
+                decoded[k, i: i + 128] = orc.decode_layer(idx[i: i + 128], sg[i: i + 128], bn, levels[m])
+            assert not got_bn[(hi - lo + 127) // 128:].any()                 # rows past the layer's end
+            wo = plan.word_offsets[m] + b0 * 32 * C
+            words = pk[0][k, wo: wo + nb * 32 * C].cpu().numpy().view(np.uint32)
+            gi, gs = orc.unpack_layer(words, hi - lo, w.bits)
+            assert np.array_equal(gi, idx) and np.array_equal(gs, sg), (m, b0, k)
+        assert np.array_equal(gbar[e0 + lo: e0 + hi].cpu().numpy(), orc.aggregate(decoded)), (m, b0)
+
+    nblk0 = (w.layer_sizes[0] + 1023) // 1024
+    for b0 in [0, 127, int(rng.integers(0, nblk0 - 4)), nblk0 - 2]:
+        check_blocks(0, b0, 2)
+    for m in [1, 7, 12, 104, Lr - 1]:
+        nb = (w.layer_sizes[m] + 1023) // 1024
+        check_blocks(m, max(0, nb - 2), min(2, nb))
+    emb = slice(plan.elem_offsets[0], plan.elem_offsets[0] + w.layer_sizes[0])
+    zero_all = (grads[:, emb] == 0).all(dim=0)
+    assert torch.equal(Y[emb][zero_all], Y_before[emb][zero_all]) and bool((gbar[emb][zero_all] == 0).all())
+    assert bool(torch.isfinite(Xh).all()) and bool(torch.isfinite(Y).all())
+
+
 # ------------------------------------------------------------------------------ config 5
 @pytest.mark.parametrize("bits", [2, 3, 4, 8])
 @pytest.mark.parametrize("K", [1, 4, 16])
