@@ -232,6 +232,11 @@ int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* coun
  *   lq_code_build   (host only, no device work): Huffman lengths for the weights (probabilities or counts,
  *                   e.g. from lq_level_probabilities / lq_symbol_counts); every symbol gets a word, and words
  *                   longer than LQ_CODE_MAX_LEN are avoided by raising the smallest weights.
+ *   lq_code_universal (host only): the word lengths of Elias' recursive code of j + 1 for level index j - the
+ *                   appendix's choice when only "smaller values are more frequent" is known, no frequencies: 1, 3,
+ *                   3, 6 x 4, 7 x 8, 11 x 16, 12 x 32 bits.  The stage sends the canonical words of these lengths,
+ *                   so the stream has the recursive code's size.  LQ_EINVAL when a word would exceed
+ *                   LQ_CODE_MAX_LEN (n > 63).
  *   lq_code_set/get: lengths host [n], n = 2^b of the layer; set refuses lengths that violate Kraft's inequality
  *                   and synchronises the device.
  * Stream of one worker: the layout's blocks of 1024 coordinates, layer after layer, each starting on a 32-bit
@@ -248,6 +253,7 @@ int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* coun
  *                   its end, sets a flag that lq_entropy_status returns (and clears); nothing faults. */
 #define LQ_CODE_MAX_LEN 12
 int lq_code_build(const double* weights, int32_t n, uint8_t* lengths);
+int lq_code_universal(int32_t n, uint8_t* lengths);
 int lq_code_set(lq_plan* plan, int32_t layer, const uint8_t* lengths, int32_t n);
 int lq_code_get(lq_plan* plan, int32_t layer, uint8_t* lengths, int32_t n);
 int64_t lq_plan_blocks(const lq_plan* plan);        /* blocks of 1024 coordinates per worker, all layers */

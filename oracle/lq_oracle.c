@@ -696,3 +696,49 @@ int64_t orc_entropy_decode_block(const uint32_t* words, int count, const uint8_t
     }
     return t;
 }
+
+/* ------------------------------------------------------------------------------------
+ * Elias' recursive ("omega") code of a positive integer (Elias 1975, cited by the appendix on
+ * the coding framework for the case where only "smaller values are more frequent" is known).
+ * Definition, written out: start from the single bit 0; while value > 1, put the binary
+ * representation of value in front and continue with value = (number of bits just written) - 1.
+ * bits_out receives the word as '0'/'1' characters (at most 63 + terminator); returns its length.
+ * orc_elias_omega_decode reads one word from a '0'/'1' string and returns the value (0 on a
+ * malformed word); *used receives the number of characters consumed.
+ * ---------------------------------------------------------------------------------- */
+int orc_elias_omega(uint64_t value, char* bits_out)
+{
+    char word[160];
+    int end = 159, start = 159;
+    word[end] = '\0';
+    word[--start] = '0';
+    if (value == 0) { bits_out[0] = '\0'; return 0; }
+    while (value > 1) {
+        int nb = 0;
+        for (uint64_t t = value; t; t >>= 1) ++nb;
+        for (int i = 0; i < nb; ++i) word[--start] = (char)('0' + (int)((value >> i) & 1u));   /* least significant bit last */
+        value = (uint64_t)(nb - 1);
+    }
+    const int len = end - start;
+    memcpy(bits_out, word + start, (size_t)len + 1);
+    return len;
+}
+
+uint64_t orc_elias_omega_decode(const char* bits, int* used)
+{
+    uint64_t n = 1;
+    int pos = 0;
+    for (;;) {
+        if (bits[pos] == '0') { ++pos; break; }
+        if (bits[pos] != '1') { if (used) *used = pos; return 0; }
+        uint64_t v = 0;
+        for (uint64_t i = 0; i <= n; ++i) {
+            const char ch = bits[pos++];
+            if (ch != '0' && ch != '1') { if (used) *used = pos; return 0; }
+            v = (v << 1) | (uint64_t)(ch - '0');
+        }
+        n = v;
+    }
+    if (used) *used = pos;
+    return n;
+}

@@ -83,6 +83,10 @@ def lib():
         L.orc_sq_norm.restype = C.c_double
         L.orc_sq_norm.argtypes = [f32p, C.c_int64]
         L.orc_qoda_update_rates.argtypes = [f32p, f32p, f32p, f32p, f32p, C.c_float, C.c_float, C.c_int64]
+        L.orc_elias_omega.restype = C.c_int
+        L.orc_elias_omega.argtypes = [C.c_uint64, C.c_char_p]
+        L.orc_elias_omega_decode.restype = C.c_uint64
+        L.orc_elias_omega_decode.argtypes = [C.c_char_p, C.POINTER(C.c_int)]
         _lib = L
     return _lib
 
@@ -240,6 +244,20 @@ def huffman_lengths(weights, max_len: int = 12) -> np.ndarray:
     ok = lib().orc_huffman_lengths(_p(w, C.c_double), w.size, max_len, _p(out, C.c_uint8))
     assert ok
     return out
+
+
+def elias_omega(value: int) -> str:
+    """Elias' recursive code word of a positive integer, as a string of '0' and '1'."""
+    buf = C.create_string_buffer(160)
+    n = lib().orc_elias_omega(C.c_uint64(int(value)), buf)
+    return buf.value.decode()[:n]
+
+
+def elias_omega_decode(bits: str):
+    """(value, characters used) of the first word in `bits`; value 0 if malformed."""
+    used = C.c_int(0)
+    v = lib().orc_elias_omega_decode(bits.encode(), C.byref(used))
+    return int(v), used.value
 
 
 def canonical_codes(lengths) -> np.ndarray:

@@ -25,7 +25,7 @@ EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan
            "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_worker_range", "lq_side_data_export",
            "lq_side_data_import", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
-           "qoda_get_scalars", "lq_code_build", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
+           "qoda_get_scalars", "lq_code_build", "lq_code_universal", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
            "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
@@ -74,6 +74,7 @@ def load_library() -> C.CDLL:
     L.qoda_get_scalars.argtypes = [vp, C.POINTER(i64), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     u8p = C.POINTER(C.c_uint8)
     L.lq_code_build.argtypes = [C.POINTER(C.c_double), i32, u8p]
+    L.lq_code_universal.argtypes = [i32, u8p]
     L.lq_code_set.argtypes = [vp, i32, u8p, i32]
     L.lq_code_get.argtypes = [vp, i32, u8p, i32]
     L.lq_plan_blocks.argtypes = [vp]; L.lq_plan_blocks.restype = i64
@@ -132,6 +133,13 @@ def lq_code_build(weights) -> List[int]:
     n = len(weights)
     w = (C.c_double * n)(*[float(x) for x in weights]); out = (C.c_uint8 * n)()
     _check(load_library().lq_code_build(w, n, out))
+    return list(out)
+
+
+def lq_code_universal(n: int) -> List[int]:
+    """Word lengths of Elias' recursive code for level indices 0..n-1 (host only)."""
+    out = (C.c_uint8 * n)()
+    _check(load_library().lq_code_universal(int(n), out))
     return list(out)
 
 

@@ -727,6 +727,28 @@ int lq_code_build(const double* weights, int32_t n, uint8_t* lengths)
     return LQ_OK;
 }
 
+int lq_code_universal(int32_t n, uint8_t* lengths)
+{
+    if (!lengths) return fail(LQ_EINVAL, "NULL argument");
+    if (n < 1 || n > kMaxLevels) return fail(LQ_EINVAL, "n must be in [1, %d]", kMaxLevels);
+    for (int j = 0; j < n; ++j) {
+        // length of the recursive code of j + 1: the closing 0, then the binary forms of the value, of its bit
+        // count minus one, and so on down to 1
+        int len = 1;
+        for (unsigned v = (unsigned)j + 1u; v > 1u;) {
+            int nb = 0;
+            for (unsigned t = v; t; t >>= 1) ++nb;
+            len += nb;
+            v = (unsigned)nb - 1u;
+        }
+        if (len > kCodeMaxLen)
+            return fail(LQ_EINVAL, "the recursive code of level index %d has %d bits, more than %d: use it with at "
+                        "most 63 levels (b <= 5)", j, len, kCodeMaxLen);
+        lengths[j] = (uint8_t)len;
+    }
+    return LQ_OK;
+}
+
 int lq_code_set(lq_plan* plan, int32_t layer, const uint8_t* lengths, int32_t n)
 {
     if (!plan || !lengths) return fail(LQ_EINVAL, "NULL argument");

@@ -58,7 +58,10 @@ def test_stream_matches_the_oracle_and_round_trips(lqm, orc, bits):
     rng = np.random.default_rng(bits)
     lengths = {}
     for m in range(plan.num_layers):
-        if m % 2 == 0:                                                # a Huffman code on some layers, the flat code on others
+        if m % 4 == 2 and bits <= 5:                                  # the universal recursive code where it fits
+            lengths[m] = lqm.lq_code_universal(n)
+            plan.lq_code_set(m, lengths[m])
+        elif m % 2 == 0:                                              # a Huffman code on some layers, the flat code on others
             lengths[m] = lqm.lq_code_build(rng.dirichlet(np.ones(n) * 0.3))
             plan.lq_code_set(m, lengths[m])
         else:

@@ -219,3 +219,11 @@ def test_exchange_assembles_all_rows_with_gloo_two_ranks(tmp_path):
         assert rec["ok"] and rec["range"] == [2 * r, 2]
         # the second message is encoded against the first; each encode is followed by one update
         assert rec["calls"] == [["quantize", 1, False], ["qoda_step"], ["quantize", 2, True], ["qoda_step"]]
+
+
+def test_universal_code_lengths_match_the_recursive_code(orc):
+    import paper_2505_14371_b200 as lqm
+    for n in (2, 4, 8, 16, 32, 63):
+        assert lqm.lq_code_universal(n) == [len(orc.elias_omega(j + 1)) for j in range(n)]
+    with pytest.raises(lqm.LqError):
+        lqm.lq_code_universal(64)                                      # its last word would have 13 bits

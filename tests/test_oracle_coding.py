@@ -75,3 +75,25 @@ def test_block_layout_by_hand_and_round_trip(orc):
         assert bits == int(l[idx].astype(int).sum() + np.count_nonzero(idx))
         i2, s2, used = orc.entropy_decode_block(words, count, l, c)
         assert used == bits and np.array_equal(i2, idx) and np.array_equal(s2, sg)
+
+
+def test_elias_recursive_code_words(orc):
+    """Elias' recursive code against the words its definition gives by hand, prefix-freeness, Kraft's inequality and
+    the round trip through the decoder."""
+    by_hand = {1: "0", 2: "100", 3: "110", 4: "101000", 7: "101110", 8: "1110000", 15: "1111110",
+               16: "10100100000", 100: "1011011001000"}
+    for v, w in by_hand.items():
+        assert orc.elias_omega(v) == w, v
+    words = [orc.elias_omega(v) for v in range(1, 300)]
+    assert sum(2.0 ** -len(w) for w in words) < 1.0
+    for i, a in enumerate(words):
+        for j, b in enumerate(words):
+            assert i == j or not b.startswith(a)
+    lens = [len(w) for w in words]
+    assert all(x <= y for x, y in zip(lens, lens[1:]))                 # smaller values never get longer words
+    stream = "".join(words[v - 1] for v in [5, 1, 299, 64, 2])
+    pos, out = 0, []
+    while pos < len(stream):
+        v, used = orc.elias_omega_decode(stream[pos:])
+        out.append(v); pos += used
+    assert out == [5, 1, 299, 64, 2]
