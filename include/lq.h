@@ -263,6 +263,14 @@ int lq_entropy_decode(lq_plan* plan, const uint32_t* stream_words, int64_t capac
                       const uint32_t* block_offsets, uint32_t* packed, void* stream);
 int lq_entropy_status(lq_plan* plan, uint32_t* host_flag);
 
+/* Ergodic average (the guarantees of Section 5 are stated for X-bar_{T+1/2} = sum_{t=1..T} X_{t+1/2} / T).
+ * qoda_set_average registers a caller-owned DEVICE array xsum [D_pad] of fp64 (16-byte aligned; NULL = off, the
+ * default) and zeroes it on `stream`; qoda_init zeroes it again.  Every following qoda_step first adds its incoming
+ * Xhalf - the point X_{t+1/2} at which the workers' dual vectors of this iteration were evaluated - to xsum, in
+ * fp64, then overwrites Xhalf as usual; after T steps xsum / T is the average (T = t - 1 from qoda_get_scalars).
+ * Costs one more pass over Xhalf and xsum (20 bytes per coordinate) per step. */
+int qoda_set_average(lq_plan* plan, double* xsum, void* stream);
+
 /* Alternative adaptive step sizes (Eq. Alt with the running sums of the appendix on the almost-sure
  * boundedness model): with q_hat in (0, 1/4], every following qoda_step uses
  *   eta_{t+1} = fp32((1 + lambda_{t-1} + mu_{t-1})^(-1/2)),  gamma_{t+1} = fp32((1 + lambda_{t-1})^(q_hat - 1/2)),
@@ -318,7 +326,8 @@ int lq_vector_norm_static(const float* v, int64_t n, int32_t q, float* norm_out,
 #define LQ_KERNEL_DECODE         5
 #define LQ_KERNEL_FIT            6
 #define LQ_KERNEL_ALT_FINALIZE   7
-#define LQ_NUM_KERNELS           8
+#define LQ_KERNEL_AVERAGE        8
+#define LQ_NUM_KERNELS           9
 int lq_profile_enable(lq_plan* plan, int32_t enable);
 int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches);
 

@@ -333,6 +333,7 @@ class OracleModel:
                                          # "bucket": one norm per 128 consecutive coordinates of a layer (Section 7.1)
         self.alt_qhat = 0.0              # > 0: the alternative rates of Eq. (Alt) with this exponent
         self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
+        self.xsum = None                 # running fp64 sum of the half iterates X_{t+1/2} (ergodic average, Section 5)
 
     # -- ENCODE side (Algorithm 1 line 12) ------------------------------------------------
     def quantize(self, grads: np.ndarray, step: int, want_hist: bool = False):
@@ -438,9 +439,11 @@ class OracleModel:
         self.S = 0.0; self.eta = np.float32(1.0); self.t = 1
         self.prev_decoded = None
         self.lam = 0.0; self.mu = 0.0; self.gamma = np.float32(1.0)
+        self.xsum = np.zeros(self.X1.shape, np.float64)
 
     def qoda_step(self) -> np.ndarray:
         """Consumes the message of the last quantize() call; returns gbar."""
+        self.xsum += self.Xhalf.astype(np.float64)      # X_{t+1/2}: where this iteration's dual vectors were evaluated
         if self.alt_qhat > 0.0:
             # eta_{t+1}, gamma_{t+1} use the sums through iteration t-1; this iteration's terms come after
             self.eta, self.gamma = alt_rates(self.lam, self.mu, self.alt_qhat)

@@ -26,11 +26,11 @@ EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan
            "lq_side_data_import", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_code_build", "lq_code_universal", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
-           "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
+           "lq_entropy_decode", "lq_entropy_status", "lq_level_probabilities", "lq_symbol_counts", "qoda_set_alt_rates", "qoda_set_average", "qoda_get_alt_scalars", "lq_get_statistics", "lq_vector_norm_static", "lq_profile_enable",
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
-                "decode", "fit", "alt_finalize"]
+                "decode", "fit", "alt_finalize", "average"]
 
 
 class LqError(RuntimeError):
@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
     L.lq_level_probabilities.argtypes = [vp, vp, vp, i32, i32, vp, vp]
     L.lq_symbol_counts.argtypes = [vp, vp, vp, vp]
     L.qoda_set_alt_rates.argtypes = [vp, C.c_double]
+    L.qoda_set_average.argtypes = [vp, vp, vp]
     L.qoda_get_alt_scalars.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double)]
     L.lq_get_statistics.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(u32)]
     L.lq_vector_norm_static.argtypes = [vp, i64, i32, vp, vp, vp]
@@ -292,6 +293,11 @@ class Plan:
         flag = C.c_uint32(0)
         _check(load_library().lq_entropy_status(self._h, C.byref(flag)))
         return flag.value
+
+    def qoda_set_average(self, xsum: Optional[torch.Tensor]) -> None:
+        """Registers (or with None removes) the fp64 running sum of the half iterates; the tensor must stay alive."""
+        _check(load_library().qoda_set_average(self._h, _ptr(xsum, torch.float64), _stream()))
+        self._xsum = xsum
 
     def qoda_set_alt_rates(self, q_hat: float) -> None:
         _check(load_library().qoda_set_alt_rates(self._h, float(q_hat)))

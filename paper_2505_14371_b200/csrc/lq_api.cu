@@ -86,6 +86,7 @@ struct lq_plan {
     uint32_t* d_code_bad = nullptr;        // [1] set by a decode that met an invalid stream
     std::vector<uint8_t> code_len;         // [L][256] host copy of the word lengths
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
+    double* xsum = nullptr;        // caller-owned running sum of the half iterates (qoda_set_average), or NULL
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
     // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
@@ -488,6 +489,8 @@ int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stre
     if (!plan || !X1 || !Y || !Xhalf) return fail(LQ_EINVAL, "NULL argument");
     LQ_ALIGNED(X1, 16); LQ_ALIGNED(Y, 16); LQ_ALIGNED(Xhalf, 16);
     LQ_CUDA(launch_qoda_init(plan->dev, X1, Y, Xhalf, (cudaStream_t)stream));
+    if (plan->xsum)
+        LQ_CUDA(cudaMemsetAsync(plan->xsum, 0, (size_t)plan->dev.padded_elems * sizeof(double), (cudaStream_t)stream));
     plan->qoda_ready = true;
     plan->stat_pending = false;
     return LQ_OK;
@@ -502,6 +505,8 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
     if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
     if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
     cudaStream_t s = (cudaStream_t)stream;
+    if (plan->xsum)                  // X_{t+1/2}, before this step overwrites it
+        LQ_CUDA(timed(plan, LQ_KERNEL_AVERAGE, s, [&] { return launch_average(plan->dev, Xhalf, plan->xsum, s); }));
     if (plan->alt_qhat > 0.0) {
         const double qh = plan->alt_qhat;
         LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_alt_scalars(plan->dev, qh, s); }));
@@ -518,6 +523,15 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
         }));
     }
     plan->stat_pending = false;
+    return LQ_OK;
+}
+
+int qoda_set_average(lq_plan* plan, double* xsum, void* stream)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    LQ_ALIGNED(xsum, 16);
+    plan->xsum = xsum;
+    if (xsum) LQ_CUDA(cudaMemsetAsync(xsum, 0, (size_t)plan->dev.padded_elems * sizeof(double), (cudaStream_t)stream));
     return LQ_OK;
 }
 

@@ -306,6 +306,26 @@ __global__ void qoda_init_kernel(PlanDev p, const float* __restrict__ X1, float*
     }
 }
 
+// xsum += Xhalf in fp64 (the running sum behind the ergodic average of the half iterates)
+__global__ void __launch_bounds__(256) average_kernel(const float* __restrict__ Xhalf, double* __restrict__ xsum, int64_t n4)
+{
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        const float4 x = __ldcs(reinterpret_cast<const float4*>(Xhalf) + i);
+        double2 a = reinterpret_cast<double2*>(xsum)[2 * i], b = reinterpret_cast<double2*>(xsum)[2 * i + 1];
+        a.x += (double)x.x; a.y += (double)x.y; b.x += (double)x.z; b.y += (double)x.w;
+        reinterpret_cast<double2*>(xsum)[2 * i] = a;
+        reinterpret_cast<double2*>(xsum)[2 * i + 1] = b;
+    }
+}
+
+cudaError_t launch_average(const PlanDev& p, const float* Xhalf, double* xsum, cudaStream_t s)
+{
+    const int64_t n4 = p.padded_elems / 4;
+    const unsigned blocks = (unsigned)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 + 1 : 148 * 16);
+    average_kernel<<<blocks, 256, 0, s>>>(Xhalf, xsum, n4);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
                           float* gbar, int mode, cudaStream_t s)

@@ -128,6 +128,7 @@ cudaError_t launch_entropy_decode(const PlanDev& p, const uint32_t* in, int64_t 
 cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s);
 cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s);
+cudaError_t launch_average(const PlanDev& p, const float* Xhalf, double* xsum, cudaStream_t s);
 cudaError_t launch_qoda_init(const PlanDev& p, const float* X1, float* Y, float* Xhalf,
                              cudaStream_t s);
 cudaError_t launch_fit(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,

@@ -49,15 +49,17 @@ def test_config2_bilinear_game_2000_iterations(lqm, orc):
     assert plan.padded_elems == D
     model = oracle_model(orc, plan)
     X1 = z1.cuda().contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    avg_gpu = torch.ones(D, dtype=torch.float64, device="cuda")          # the library's running sum of X_{t+1/2}
+    plan.qoda_set_average(avg_gpu)
     plan.qoda_init(X1, Y, Xh)
     model.qoda_init(z1.numpy())
     pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
     R = float(np.linalg.norm(z1.numpy().astype(np.float64)))
-    avg_gpu = torch.zeros(D, dtype=torch.float64, device="cuda"); avg_orc = np.zeros(D)
+    avg_orc = np.zeros(D)
     gaps = {}; near = 0; first_bad = None
     for t in range(1, T + 1):
         noise = W.bilinear_noise(t, K, D)                                   # host-drawn, shared by both sides
-        avg_gpu += Xh.double(); avg_orc += model.Xhalf
+        avg_orc += model.Xhalf
         V_gpu = (operator(Xh)[None, :] + noise.cuda()).contiguous()
         F_orc = operator(torch.from_numpy(model.Xhalf).cuda()).cpu().numpy()
         V_orc = F_orc[None, :] + noise.numpy()
@@ -92,6 +94,7 @@ def test_config2_bilinear_game_2000_iterations(lqm, orc):
     assert first_bad is None, f"first differing message at (step, coords, words) = {first_bad}"
     assert near < 1e-5 * K * D * T
     assert _rel((avg_gpu / T).cpu().numpy(), avg_orc / T) <= 1e-5
+    assert np.array_equal(avg_orc, model.xsum)
     assert gaps[2000] < 0.5 * gaps[100] and gaps[100] < gaps[10]
 
 

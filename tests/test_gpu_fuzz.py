@@ -53,6 +53,8 @@ def test_random_plan_against_the_oracle(orc, case):
     g = torch.Generator(device="cuda").manual_seed(case)
     X1 = (torch.randn(plan.padded_elems, generator=g, device="cuda") * 0.1).contiguous()
     Y = torch.empty_like(X1); Xh = torch.empty_like(X1); X = torch.empty_like(X1); gbar = torch.empty_like(X1)
+    xsum = torch.full((plan.padded_elems,), 7.0, dtype=torch.float64, device="cuda")
+    plan.qoda_set_average(xsum)                                  # zeroed here and again by qoda_init
     plan.qoda_init(X1, Y, Xh); model.qoda_init(to_unpadded(plan, X1))
     pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
     off = plan.elem_offsets
@@ -104,6 +106,7 @@ def test_random_plan_against_the_oracle(orc, case):
             assert abs(S - model.S) <= 1e-12 * max(model.S, 1e-300), tag
         for got, want in [(Y, model.Y), (Xh, model.Xhalf), (X, model.X)]:
             assert _close(to_unpadded(plan, got), want, 1e-6), tag
+        assert _close(to_unpadded(plan, xsum), model.xsum, 1e-6), tag      # running sum of X_{s+1/2}, s <= t
         if use_hist and rng.random() < 0.7:                      # refit from this step's histograms
             plan.lq_fit_levels(hist, nm[c], K)
             h = ref["hist"]
