@@ -112,7 +112,9 @@ int lq_set_norm_scope(lq_plan* plan, int32_t scope);
  * rows of packed and norms in (an all-gather), and their per-(worker, layer) side data - the step-size statistic
  * that qoda_step consumes, the bucket scope's fit weights, the flags - with the two calls below, before
  * lq_decode_aggregate / qoda_step / lq_fit_levels, which always cover all K workers.  Default range: (0, K).
- * LQ_EINVAL if the range does not lie inside [0, K). */
+ * A plan keeps track of one stream of messages (level tables and zero-row masks of the previous one), so choose
+ * the range once, before the first lq_quantize_pack; after a later change the next lq_quantize_pack must start a
+ * new stream (prev_packed = NULL, else LQ_ESTATE).  LQ_EINVAL if the range does not lie inside [0, K). */
 int lq_set_worker_range(lq_plan* plan, int32_t first_worker, int32_t count);
 /* Copies the plan's per-(worker, layer) side data to / from DEVICE arrays of shape [K][L] on `stream`
  * (sq_diff fp64, 8-byte aligned; layer_weight fp32; flags u32; any pointer may be NULL = skip).  Export after

@@ -89,6 +89,7 @@ struct lq_plan {
     double* xsum = nullptr;        // caller-owned running sum of the half iterates (qoda_set_average), or NULL
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
+    bool masks_known = false;              // d_row_mask[mask_cur] describes the last message of the current worker range
     // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
     struct ProfRec { int id; cudaEvent_t a, b; };
     bool profiling = false;
@@ -365,6 +366,9 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     if ((prev_packed == nullptr) != (prev_norms == nullptr))
         return fail(LQ_EINVAL, "prev_packed and prev_norms must both be given or both be NULL");
     if (prev_packed == packed) return fail(LQ_EINVAL, "prev_packed must not alias packed");
+    if (prev_packed && plan->have_message && !plan->masks_known)
+        return fail(LQ_ESTATE, "the worker range changed since the plan's last message: the first message of the new "
+                    "range has no previous message (pass prev_packed = NULL)");
     LQ_ALIGNED(grads, 16); LQ_ALIGNED(packed, 4); LQ_ALIGNED(norms, 4); LQ_ALIGNED(hist, 4);
     LQ_ALIGNED(prev_packed, 4); LQ_ALIGNED(prev_norms, 4);
     if (plan->dev.num_layers == 0) return LQ_OK;
@@ -382,7 +386,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
         plan->prev = plan->cur;
     }
     // the masks written now describe this message; the ones of the last call describe prev_packed
-    plan->dev.row_mask_prev = plan->have_message ? plan->d_row_mask[plan->mask_cur] : nullptr;
+    plan->dev.row_mask_prev = (plan->have_message && plan->masks_known) ? plan->d_row_mask[plan->mask_cur] : nullptr;
     plan->mask_cur = plan->have_message ? 1 - plan->mask_cur : plan->mask_cur;
     plan->dev.row_mask = plan->d_row_mask[plan->mask_cur];
     const PlanDev& d = plan->dev;
@@ -395,6 +399,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
         }));
         LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_bucket_finalize(d, s); }));
         plan->have_message = true;
+        plan->masks_known = true;          // (no masks in this scope: the flag also marks an unbroken stream of messages)
         plan->stat_pending = true;
         return LQ_OK;
     }
@@ -406,6 +411,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     }));
     LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_stat_finalize(d, s); }));
     plan->have_message = true;
+    plan->masks_known = true;
     plan->stat_pending = true;
     return LQ_OK;
 }
@@ -554,6 +560,8 @@ int lq_set_worker_range(lq_plan* plan, int32_t first_worker, int32_t count)
     if (first_worker < 0 || count < 1 || first_worker > plan->dev.num_workers - count)
         return fail(LQ_EINVAL, "worker range [%d, %d) is not inside [0, %d)", first_worker, first_worker + count,
                     plan->dev.num_workers);
+    if (first_worker != plan->dev.worker0 || count != plan->dev.worker_count)
+        plan->masks_known = false;         // the stored zero-row masks describe another set of workers' last input
     plan->dev.worker0 = first_worker;
     plan->dev.worker_count = count;
     return LQ_OK;

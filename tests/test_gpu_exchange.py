@@ -40,3 +40,23 @@ def test_two_ranks_equal_one_process(tmp_path, scope):
         got = np.load(tmp_path / f"rank{r}.npz")
         for key in want:
             assert np.array_equal(got[key], want[key]), (r, key)
+
+
+def test_changing_the_range_restarts_the_message_stream():
+    import torch
+    import paper_2505_14371_b200 as lqm
+    lqm.load_library()
+    plan = lqm.Plan([5000], 4, 2, 4, 3)
+    grads = torch.randn((4, plan.padded_elems), device="cuda")
+    a, b = plan.empty_packed(), plan.empty_packed(); na, nb = plan.empty_norms(), plan.empty_norms()
+    plan.lq_quantize_pack(grads, 1, a, na)
+    plan.lq_set_worker_range(2, 2)
+    with pytest.raises(lqm.LqError):
+        plan.lq_quantize_pack(grads[2:4].contiguous(), 2, b, nb, prev_packed=a, prev_norms=na)
+    b.copy_(a); nb.copy_(na)
+    plan.lq_quantize_pack(grads[2:4].contiguous(), 1, b, nb)     # same step, same workers: the same rows come out
+    torch.cuda.synchronize()
+    assert torch.equal(a, b) and torch.equal(na, nb)
+    plan.lq_quantize_pack(grads[2:4].contiguous(), 2, a, na, prev_packed=b, prev_norms=nb)   # the stream continues
+    with pytest.raises(lqm.LqError):
+        plan.lq_set_worker_range(3, 2)
