@@ -59,9 +59,6 @@ __device__ __forceinline__ uint32_t shr(uint32_t x)
 #ifndef LQ_MUL_RHO
 #define LQ_MUL_RHO 1
 #endif
-#ifndef LQ_MUL_SIGN
-#define LQ_MUL_SIGN 0
-#endif
 #ifndef LQ_MUL_LUT
 #define LQ_MUL_LUT 0
 #endif
@@ -75,6 +72,13 @@ __device__ __forceinline__ uint32_t add8_if_ge(uint32_t x, float a, float b)
 __device__ __forceinline__ uint32_t add8_if_lt(uint32_t x, float a, float b)
 {
     asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(x) : "f"(a), "f"(b));
+    return x;
+}
+
+// x + 4 when v < 0 (so neither zero sets the sign bit of a symbol), else x
+__device__ __forceinline__ uint32_t add4_if_negative(uint32_t x, float v)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %1, 0f00000000;\n\t@p add.u32 %0, %0, 4;\n\t}" : "+r"(x) : "f"(v));
     return x;
 }
 
@@ -317,9 +321,6 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
         if (live) {
             cp_async_wait<kRingRows - 1>();
             v = c.ring_ptr[32 * j];
-            // -0 becomes +0 (the sign of a coordinate is v < 0); every other value is unchanged
-            v.x = __fadd_rn(v.x, 0.0f); v.y = __fadd_rn(v.y, 0.0f);
-            v.z = __fadd_rn(v.z, 0.0f); v.w = __fadd_rn(v.w, 0.0f);
         }
         const float vv[4] = {v.x, v.y, v.z, v.w};
         if (live) {
@@ -328,7 +329,6 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int pp = 4 * j + e;
-                const uint32_t bits = __float_as_uint(vv[e]);
                 // u <= 1 + 2^-23 always (N >= |v| and one rounding each in 1/N and the product), and
                 // such a u behaves exactly like u = 1 below, so the min(u, 1) of the definition is not needed
                 const float u = __fmul_rn(fabsf(vv[e]), r);
@@ -355,7 +355,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 const float f = __uint_as_float(shr<9, LQ_MUL_RHO>(x[e]) + 0x3F800000u);
                 const float t = __fmaf_rn(f, den, -den);
                 const uint32_t i8 = add8_if_lt(t8, t, num);
-                const uint32_t sym4 = i8 | (shr<29, LQ_MUL_SIGN>(bits) & 4u);     // 4 * (2 * idx + sign)
+                const uint32_t sym4 = add4_if_negative(i8, vv[e]);                // 4 * (2 * idx + sign), sign = (v < 0)
                 put_symbol4<C>(cw, pp, sym4);
 
                 if (kHist) {
