@@ -46,23 +46,6 @@ struct QuantSmem {
     uint8_t rows_prev[kTileBlocks];  // the same for the input behind the previous message
 };
 
-// x >> K for a constant K.  kMul writes it as the high half of a multiplication, which runs on the
-// multiply-add pipe instead of the integer/logic pipe.
-template <int K, bool kMul>
-__device__ __forceinline__ uint32_t shr(uint32_t x)
-{
-    if (!kMul) return x >> K;
-    uint32_t d;
-    asm("mul.hi.u32 %0, %1, %2;" : "=r"(d) : "r"(x), "r"(1u << (32 - K)));
-    return d;
-}
-#ifndef LQ_MUL_RHO
-#define LQ_MUL_RHO 1
-#endif
-#ifndef LQ_MUL_LUT
-#define LQ_MUL_LUT 0
-#endif
-
 // x + 8 when a >= b (resp. a < b), else x: one compare and one predicated add
 __device__ __forceinline__ uint32_t add8_if_ge(uint32_t x, float a, float b)
 {
@@ -335,7 +318,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 const uint32_t ub = __float_as_uint(u);
                 uint32_t t8;
                 if (kFast) {
-                    const uint32_t off = shr<16, LQ_MUL_LUT>(max(ub, kLutClamp)) & ~7u;
+                    const uint32_t off = (max(ub, kLutClamp) >> 16) & ~7u;
                     const uint2 en = *reinterpret_cast<const uint2*>(lut_b + off);
                     t8 = add8_if_ge(en.x, u, __uint_as_float(en.y));
                 } else {
@@ -352,7 +335,8 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 const float num = __fsub_rn(u, ld.x);
                 // rho = (x >> 9) * 2^-23; f = 1 + rho is built from the bits, and fma(f, den, -den)
                 // rounds the exact product rho * den once, like the plain multiplication
-                const float f = __uint_as_float(shr<9, LQ_MUL_RHO>(x[e]) + 0x3F800000u);
+                // (one funnel shift: the 64-bit value {0x7F, x} moved right by 9 is (x >> 9) | 0x3F800000)
+                const float f = __uint_as_float(__funnelshift_r(x[e], 0x7Fu, 9));
                 const float t = __fmaf_rn(f, den, -den);
                 const uint32_t i8 = add8_if_lt(t8, t, num);
                 const uint32_t sym4 = add4_if_negative(i8, vv[e]);                // 4 * (2 * idx + sign), sign = (v < 0)
