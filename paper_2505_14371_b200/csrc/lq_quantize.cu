@@ -363,6 +363,11 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
                 stat = fma(dd, dd, stat);
             }
         }
+        if (kHist && !kBucket && !live && lane == 0) {
+            // an all-zero row of a layer with a norm: its coordinates have u = 0 and count in the first bin
+            const int64_t rem = c.size - (blk * kBlockCoords + 128 * j);
+            if (rem > 0) atomicAdd(&sm.hist[0], (uint32_t)(rem < 128 ? rem : 128));
+        }
         if (next && ((next_rows >> j) & 1u)) cp_async16(c.ring + 512u * j, next + 128 * j, 16);
         cp_async_commit();
     }
@@ -418,6 +423,10 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
             const int64_t woff = blk * (int64_t)C * 32 + c.lane;
 #pragma unroll
             for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, 0u);
+            if (kHist && c.lane == 0) {                   // its coordinates all have u = 0
+                const int64_t rem = c.size - blk * kBlockCoords;
+                atomicAdd(&sm.hist[0], (uint32_t)(rem < kBlockCoords ? rem : kBlockCoords));
+            }
             continue;
         }
         if (!primed) {
@@ -448,6 +457,10 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
             const int64_t woff = (tile.block0 + nb) * (int64_t)C * 32 + c.lane;
 #pragma unroll
             for (int w = 0; w < C; ++w) __stcs(out + woff + w * 32, 0u);
+            if (kHist && c.lane == 0) {
+                const int64_t rem = c.size - (tile.block0 + nb) * kBlockCoords;
+                atomicAdd(&sm.hist[0], (uint32_t)(rem < kBlockCoords ? rem : kBlockCoords));
+            }
             nb += kQWarps;
         }
         const bool has_next = nb < tile.nblocks;
@@ -499,10 +512,9 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     if (kHist)
         for (int i = threadIdx.x; i < LQ_HIST_STRIDE; i += blockDim.x) sm.hist[i] = 0;
     if (threadIdx.x < tile.nblocks) {
-        // with a histogram every coordinate counts, zero or not, so every row is fetched; a previous
-        // message whose masks are unknown is taken as nonzero everywhere
+        // a previous message whose masks are unknown is taken as nonzero everywhere
         const int64_t mb = (int64_t)k * p.total_blocks + L.block_off + tile.block0 + threadIdx.x;
-        sm.rows_cur[threadIdx.x] = (kHist || kBucket) ? (uint8_t)0xff : p.row_mask[mb];
+        sm.rows_cur[threadIdx.x] = kBucket ? (uint8_t)0xff : p.row_mask[mb];
         sm.rows_prev[threadIdx.x] = !prev_packed ? (uint8_t)0
                                     : ((p.row_mask_prev && !kBucket) ? p.row_mask_prev[mb] : (uint8_t)0xff);
     }
