@@ -225,6 +225,10 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     while ((1 << d.sub_shift) < d.sub_tiles) ++d.sub_shift;
     d.padded_elems = elem; d.packed_words = word; d.total_blocks = blocks;
     d.seed_lo = (uint32_t)seed; d.seed_hi = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 8; ++r) {
+        d.rk0[r] = d.seed_lo + (uint32_t)(r + 2) * 0x9E3779B9u;
+        d.rk1[r] = d.seed_hi + (uint32_t)(r + 2) * 0xBB67AE85u;
+    }
 
     cudaError_t e = cudaGetDevice(&p->device);
     const size_t KL = (size_t)num_workers * (size_t)(num_layers ? num_layers : 1);

@@ -69,6 +69,8 @@ struct PlanDev {
     int64_t padded_elems; // D_pad
     int64_t packed_words; // W
     uint32_t seed_lo, seed_hi;
+    uint32_t rk0[8], rk1[8];  // Philox keys of rounds 2..9 (seed words plus multiples of the Weyl constants): kernels
+                              // read them straight from the parameter bank
     double* norm_partial; // [K][num_tiles * sub_tiles]
     double* stat_partial; // [K][num_tiles]
     double* sq_diff;      // [K][L]

@@ -81,7 +81,6 @@ struct PhiloxConsts {
     uint32_t c1;     // lo(M1 worker) ^ (k0 + W0)       (round 1: c0'' = hi(M1 c2') ^ c1)
     uint32_t c2;     // hi(M0 a0) ^ (k1 + W1)           (round 1: c2'' = lo(M0 c0) ^ c2)
     uint32_t l0;     // lo(M0 a0)                       (round 1: c3'')
-    uint32_t rk0[8], rk1[8];   // the keys of rounds 2..9
 };
 
 __device__ __forceinline__ PhiloxConsts philox_fold(uint32_t layer, uint32_t worker, uint32_t step,
@@ -95,15 +94,12 @@ __device__ __forceinline__ PhiloxConsts philox_fold(uint32_t layer, uint32_t wor
     pc.c1 = (uint32_t)p1 ^ (k0 + 0x9E3779B9u);
     pc.c2 = (uint32_t)(q0 >> 32) ^ (k1 + 0xBB67AE85u);
     pc.l0 = (uint32_t)q0;
-#pragma unroll
-    for (int r = 0; r < 8; ++r) {
-        pc.rk0[r] = k0 + (uint32_t)(r + 2) * 0x9E3779B9u;
-        pc.rk1[r] = k1 + (uint32_t)(r + 2) * 0xBB67AE85u;
-    }
     return pc;
 }
 
-__device__ __forceinline__ void philox4x32_10_folded(uint32_t ctr0, const PhiloxConsts& pc, uint32_t (&out)[4])
+// (the keys of rounds 2..9 depend on the seed only and come from the kernel's parameters)
+__device__ __forceinline__ void philox4x32_10_folded(uint32_t ctr0, const PhiloxConsts& pc, const PlanDev& p,
+                                                     uint32_t (&out)[4])
 {
     // rounds 0 and 1 with their constant halves folded
     const uint64_t p0 = (uint64_t)0xD2511F53u * ctr0;
@@ -117,8 +113,8 @@ __device__ __forceinline__ void philox4x32_10_folded(uint32_t ctr0, const Philox
     for (int r = 0; r < 8; ++r) {
         const uint64_t q0 = (uint64_t)0xD2511F53u * c0;
         const uint64_t q1 = (uint64_t)0xCD9E8D57u * c2;
-        const uint32_t n0 = (uint32_t)(q1 >> 32) ^ c1 ^ pc.rk0[r];
-        const uint32_t n2 = (uint32_t)(q0 >> 32) ^ c3 ^ pc.rk1[r];
+        const uint32_t n0 = (uint32_t)(q1 >> 32) ^ c1 ^ p.rk0[r];
+        const uint32_t n2 = (uint32_t)(q0 >> 32) ^ c3 ^ p.rk1[r];
         c1 = (uint32_t)q1;
         c3 = (uint32_t)q0;
         c0 = n0;
@@ -247,7 +243,7 @@ __device__ __forceinline__ void bucket_norms8(const float4* ring_ptr, int q, int
 // says which rows may be nonzero in the previous message.  Returns this lane's statistic term.
 // In bucket scope the value tables hold the plain signed levels and every row brings its own norm.
 template <int B, bool kFast, bool kHist, bool kBucket>
-__device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const WarpCtx& c,
+__device__ __forceinline__ double quantize_block(const PlanDev& p, const PhiloxConsts& pc, const WarpCtx& c,
                                                  int64_t blk, uint32_t rows, uint32_t prev_rows,
                                                  const float* __restrict__ next, uint32_t next_rows,
                                                  uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
@@ -308,7 +304,7 @@ __device__ __forceinline__ double quantize_block(const PhiloxConsts& pc, const W
         const float vv[4] = {v.x, v.y, v.z, v.w};
         if (live) {
             uint32_t x[4];
-            philox4x32_10_folded(ctr0 + 32 * j, pc, x);
+            philox4x32_10_folded(ctr0 + 32 * j, pc, p, x);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int pp = 4 * j + e;
@@ -407,7 +403,7 @@ __device__ __forceinline__ double zeroed_tile(const Tile& tile, int lane, uint32
 // in the input behind the previous message is an all-zero piece of message that adds nothing to the
 // statistic: its words are stored and nothing is read.
 template <int B, bool kFast, bool kHist, bool kBucket>
-__device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const WarpCtx& c, const Tile& tile,
+__device__ __forceinline__ double quantize_tile(const PlanDev& p, const PhiloxConsts& pc, const WarpCtx& c, const Tile& tile,
                                                 uint32_t* __restrict__ out,
                                                 const uint32_t* __restrict__ prev, QuantSmem& sm, BucketCtx& bk)
 {
@@ -467,7 +463,7 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
         const int64_t nblk = tile.block0 + nb;
         const uint32_t next_rows = has_next ? sm.rows_cur[nb] : 0u;
         const float* next = (has_next && nblk < nfull) ? c.g + nblk * kBlockCoords + 4 * c.lane : nullptr;
-        stat += quantize_block<B, kFast, kHist, kBucket>(pc, c, blk, rows, pmask, next, next_rows, out, pw, sm, bk, prev_norm8);
+        stat += quantize_block<B, kFast, kHist, kBucket>(p, pc, c, blk, rows, pmask, next, next_rows, out, pw, sm, bk, prev_norm8);
         primed = has_next;
         if (has_next && nblk >= nfull) issue_ragged_block(c, nblk);   // the layer's last, partial block
         b = nb - kQWarps;                                             // the loop's increment lands on nb
@@ -477,7 +473,7 @@ __device__ __forceinline__ double quantize_tile(const PhiloxConsts& pc, const Wa
 }
 
 template <bool kHist, bool kBucket>
-__global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
+__global__ void __launch_bounds__(kQThreads, kBucket ? 3 : 4) quantize_pack_kernel(
     PlanDev p, const float* __restrict__ grads, uint32_t step, uint32_t* __restrict__ packed,
     const float* __restrict__ norms, float* __restrict__ bucket_norms, uint32_t* __restrict__ hist,
     const uint32_t* __restrict__ prev_packed, const float* __restrict__ prev_norms,
@@ -542,8 +538,8 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_kernel(
     switch (zeroed ? -L.bits : L.bits * 2 + (fast ? 1 : 0)) {
 #define LQ_CASE(BB)                                                                              \
     case -BB:        stat = zeroed_tile<BB>(tile, lane, out, prev, sm); break;                   \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist, kBucket>(pc, c, tile, out, prev, sm, bk); break;  \
-    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist, kBucket>(pc, c, tile, out, prev, sm, bk); break;
+    case 2 * BB:     stat = quantize_tile<BB, false, kHist, kBucket>(p, pc, c, tile, out, prev, sm, bk); break;  \
+    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist, kBucket>(p, pc, c, tile, out, prev, sm, bk); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
