@@ -293,10 +293,21 @@ def run_gpu(args) -> None:
         host_out = torch.empty(Xh.shape, dtype=torch.float32, pin_memory=True)
         e2e_steps = max(1, min(args.steps, 5))
 
+        # the result travels back on a second stream, so that it shares the link with the next step's input
+        # (PCIe is full duplex); the next update waits for that copy before it overwrites the iterate
+        back = torch.cuda.Stream(device=dev)
+        done_step, done_copy = torch.cuda.Event(), torch.cuda.Event()
+        done_copy.record()
+
         def e2e_step():
             grads.copy_(host_grads, non_blocking=True)
+            torch.cuda.current_stream().wait_event(done_copy)
             step()
-            host_out.copy_(Xh, non_blocking=True)
+            done_step.record()
+            with torch.cuda.stream(back):
+                back.wait_event(done_step)
+                host_out.copy_(Xh, non_blocking=True)
+                done_copy.record()
 
         e2e_step(); barrier()
         e0.record()
