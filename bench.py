@@ -284,6 +284,29 @@ def run_gpu(args) -> None:
     prof = plan.lq_profile_read()
     plan.lq_profile_enable(False)
     ms = aggregate_over_ranks(local_ms, world, dev)
+    graph_ms = None
+    if args.graph and ex is None:
+        # two iterations recorded once (messages and masks are double-buffered), replayed steps / 2 times; the step
+        # index comes from the plan's device-side counter, so nothing in the recording changes between replays
+        def auto_step():
+            state["t"] += 1
+            c, p = state["t"] % 2, (state["t"] + 1) % 2
+            plan.lq_quantize_pack(grads, pkg.STEP_AUTO, packed[c], norms[c], prev_packed=packed[p], prev_norms=norms[p])
+            plan.qoda_step(packed[c], norms[c], X1, Y, Xh)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            auto_step(); auto_step()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        reps = max(1, args.steps // 2)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_ms = aggregate_over_ranks(e0.elapsed_time(e1) / (2 * reps), world, dev)
 
     # ---- end to end: pinned host gradients in, new iterate out ------------------------------
     e2e = None
@@ -390,6 +413,9 @@ def run_gpu(args) -> None:
                        "multi_gpu": "K workers shared out over the ranks, messages by all-gather" if args.exchange
                                     else "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "calls": calls}
+    if graph_ms is not None:
+        line["cuda_graph"] = {"ms_per_step": graph_ms, "value": whole_job_value(4.0 * K * D * share / 1e9, world, graph_ms),
+                              "note": "the same two calls per step, two steps recorded once and replayed"}
     if cpu:
         line["cpu_baseline"] = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
     print(json.dumps(line), flush=True)
@@ -477,6 +503,8 @@ def main() -> None:
     ap.add_argument("--workload", default="transformer_xl")
     ap.add_argument("--norm-scope", default="layer", choices=["layer", "global", "bucket"],
                     help="layer: one norm per layer (the headline configuration); bucket: one per 128 coordinates")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="skip the extra timing of the step replayed from a CUDA graph (reported under cuda_graph)")
     ap.add_argument("--exchange", action="store_true",
                     help="share the K workers out over the ranks and exchange the messages by all-gather (default: "
                          "every rank runs the whole K-worker job on its own data)")

@@ -161,7 +161,15 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
  *     that call's input were all zero and does not read the corresponding words again.
  *   prev_packed must not alias packed.
  *   The sign of a coordinate is (v < 0): +0 and -0 both give symbol 0, so rows of zeros (of either
- *   sign) become all-zero words; such rows are detected by the norm pass and not read again. */
+ *   sign) become all-zero words; such rows are detected by the norm pass and not read again.
+ *   step = LQ_STEP_AUTO: the kernels take the step index from the plan's iteration counter on the device (the
+ *   t of qoda_get_scalars, advanced by every qoda_step, 1 after qoda_init) instead of from the host.  Then no
+ *   argument of an iteration changes from one pair of iterations to the next, so a caller may record
+ *   [lq_quantize_pack, qoda_step] x 2 (two iterations, because messages and masks are double-buffered) into a
+ *   CUDA graph on its stream and replay it: every call only enqueues work on `stream` and keeps its plan-side
+ *   bookkeeping on the host, where the replays leave it as the recording did.  A level change (lq_set_levels,
+ *   lq_fit_levels) needs a new recording, and profiling (lq_profile_enable) must be off while recording. */
+#define LQ_STEP_AUTO 0xFFFFFFFFu
 int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t* packed,
                      float* norms, uint32_t* hist, const uint32_t* prev_packed,
                      const float* prev_norms, void* stream);

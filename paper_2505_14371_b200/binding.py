@@ -20,6 +20,7 @@ NUM_BINS = 386
 HIST_STRIDE = 512
 STATUS_ZERO_NORM = 1
 STATUS_NONFINITE = 2
+STEP_AUTO = 0xFFFFFFFF          # lq_quantize_pack: take the step index from the plan's device-side iteration counter
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
            "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_worker_range", "lq_side_data_export",

@@ -530,6 +530,7 @@ __global__ void __launch_bounds__(kQThreads, kBucket ? 3 : 4) quantize_pack_kern
         bk.prev_bn = prev_norms ? prev_norms + bo : nullptr;
         bk.bn_out = bucket_norms + bo;
     }
+    if (step == LQ_STEP_AUTO) step = (uint32_t)p.scalars->t;      // the plan's own iteration counter (graph replays)
     const PhiloxConsts pc = philox_fold((uint32_t)layer, (uint32_t)k, step, p.seed_lo, p.seed_hi);
     uint32_t* out = packed + (int64_t)k * p.packed_words + L.word_off;
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
