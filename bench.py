@@ -391,7 +391,7 @@ def run_gpu(args) -> None:
                 "note": "achieved = algorithmic bytes per launch / CUDA-event time; the encoder skips rows that the "
                         "norm pass found all zero, so its DRAM traffic is below its algorithmic bytes"}
     qp_ms = sum(kern[n]["avg_ms"] for n in ("norm_partial", "norm_finalize", "quantize_pack", "stat_finalize") if n in kern)
-    st_ms = sum(kern[n]["avg_ms"] for n in ("qoda_scalars", "decode") if n in kern)
+    st_ms = sum(kern[n]["avg_ms"] for n in ("qoda_scalars", "block_live", "decode") if n in kern)
     calls = {"lq_quantize_pack": {"ms": qp_ms, "fp32_in_gbs": 4.0 * K * D / qp_ms / 1e6,
                                   "algorithmic_gbs": qp_alg / qp_ms / 1e6,
                                   "frac_of_peak": qp_alg / qp_ms / 1e6 / peak,

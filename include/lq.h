@@ -212,6 +212,11 @@ int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stre
  *   gbar = mean of the K decoded messages,  Y_{t+1} = Y_t - gbar,
  *   X_{t+1} = fma(eta_{t+1}, Y_{t+1}, X_1),  X_{t+3/2} = fma(-gamma_{t+1}, gbar, X_{t+1}).
  * One fused pass: each packed message is read once.
+ * qoda_step consumes the message of the plan's last lq_quantize_pack (whose statistic it uses; LQ_ESTATE if there
+ * is no new one).  When `packed` is the very buffer that call wrote for all K workers (layer or global scope),
+ * the buffer must still hold that message: blocks the encoder knows to be all zero are not read again, and where no
+ * worker sent anything Y is left as it is.  A message at another address, and one assembled from several worker
+ * ranges, is read in full.
  *   packed dev [K][W], norms dev [K][L], X1 dev [D_pad] in;  Y dev [D_pad] in/out;
  *   Xhalf dev [D_pad] out (X_{t+3/2});  X_opt, gbar_opt: NULL or dev [D_pad] out. */
 int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1,
@@ -337,7 +342,8 @@ int lq_vector_norm_static(const float* v, int64_t n, int32_t q, float* norm_out,
 #define LQ_KERNEL_FIT            6
 #define LQ_KERNEL_ALT_FINALIZE   7
 #define LQ_KERNEL_AVERAGE        8
-#define LQ_NUM_KERNELS           9
+#define LQ_KERNEL_BLOCK_LIVE     9
+#define LQ_NUM_KERNELS           10
 int lq_profile_enable(lq_plan* plan, int32_t enable);
 int lq_profile_read(lq_plan* plan, double* total_ms, int64_t* launches);
 

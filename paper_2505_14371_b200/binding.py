@@ -31,7 +31,7 @@ EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan
            "lq_profile_read",
            "lq_error_string", "lq_last_error"]
 KERNEL_NAMES = ["norm_partial", "norm_finalize", "quantize_pack", "stat_finalize", "qoda_scalars",
-                "decode", "fit", "alt_finalize", "average"]
+                "decode", "fit", "alt_finalize", "average", "block_live"]
 
 
 class LqError(RuntimeError):

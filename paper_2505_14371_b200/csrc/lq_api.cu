@@ -87,6 +87,7 @@ struct lq_plan {
     std::vector<uint8_t> code_len;         // [L][256] host copy of the word lengths
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
     double* xsum = nullptr;        // caller-owned running sum of the half iterates (qoda_set_average), or NULL
+    const uint32_t* last_packed = nullptr;   // where the last lq_quantize_pack wrote its message
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
     bool masks_known = false;              // d_row_mask[mask_cur] describes the last message of the current worker range
@@ -107,6 +108,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
     cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.block_live);
     cudaFree(p->dev.energy_partial); cudaFree(p->dev.flag_partial); cudaFree(p->dev.layer_weight);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
     for (auto e : p->prof_pool) cudaEventDestroy(e);
@@ -133,6 +135,17 @@ cudaError_t timed(lq_plan* p, int id, cudaStream_t s, F&& launch)
     cudaEventRecord(b, s);
     p->prof_recs.push_back({id, a, b});
     return e;
+}
+
+// Per block the bitmask of workers that sent anything, if `packed` is the message the plan's last lq_quantize_pack
+// wrote for all K <= 32 workers in the layer or global scope (the decoder then leaves all-zero blocks unread);
+// otherwise nullptr.
+const uint32_t* message_masks(const lq_plan* p, const uint32_t* packed)
+{
+    const PlanDev& d = p->dev;
+    if (!p->have_message || !p->masks_known || d.bucket_norm || packed != p->last_packed) return nullptr;
+    if (d.worker0 != 0 || d.worker_count != d.num_workers || d.num_workers > 32) return nullptr;
+    return d.block_live;
 }
 
 template <typename T>
@@ -249,6 +262,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&d.rnorm, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.status, KL);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_total, KL);
+    if (e == cudaSuccess) e = dev_alloc_zero(&d.block_live, (size_t)(blocks ? blocks : 1));
     if (e == cudaSuccess) e = dev_alloc_zero(&d.energy_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.flag_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.layer_weight, KL);
@@ -416,6 +430,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_stat_finalize(d, s); }));
     plan->have_message = true;
     plan->masks_known = true;
+    plan->last_packed = packed;
     plan->stat_pending = true;
     return LQ_OK;
 }
@@ -489,7 +504,7 @@ int lq_decode_aggregate(const lq_plan* plan, const uint32_t* packed, const float
     lq_plan* mp = const_cast<lq_plan*>(plan);      // the profiler's bookkeeping is not plan state
     LQ_CUDA(timed(mp, LQ_KERNEL_DECODE, s, [&] {
         return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], nullptr, nullptr,
-                             nullptr, nullptr, gbar, 0, s);
+                             nullptr, nullptr, gbar, 0, nullptr, s);
     }));
     return LQ_OK;
 }
@@ -515,6 +530,9 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
     if (!plan->qoda_ready) return fail(LQ_ESTATE, "qoda_step before qoda_init");
     if (!plan->stat_pending) return fail(LQ_ESTATE, "qoda_step needs a new lq_quantize_pack message");
     cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t* live = message_masks(plan, packed);
+    if (live)                        // folds the K workers' zero-row masks into one word per block
+        LQ_CUDA(timed(plan, LQ_KERNEL_BLOCK_LIVE, s, [&] { return launch_block_live(plan->dev, s); }));
     if (plan->xsum)                  // X_{t+1/2}, before this step overwrites it
         LQ_CUDA(timed(plan, LQ_KERNEL_AVERAGE, s, [&] { return launch_average(plan->dev, Xhalf, plan->xsum, s); }));
     if (plan->alt_qhat > 0.0) {
@@ -522,14 +540,14 @@ int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const f
         LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_alt_scalars(plan->dev, qh, s); }));
         LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
             return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
-                                 gbar_opt, 2, s);
+                                 gbar_opt, 2, live, s);
         }));
         LQ_CUDA(timed(plan, LQ_KERNEL_ALT_FINALIZE, s, [&] { return launch_alt_finalize(plan->dev, s); }));
     } else {
         LQ_CUDA(timed(plan, LQ_KERNEL_QODA_SCALARS, s, [&] { return launch_qoda_scalars(plan->dev, s); }));
         LQ_CUDA(timed(plan, LQ_KERNEL_DECODE, s, [&] {
             return launch_decode(plan->dev, packed, norms, plan->d_levels_enc[plan->cur], X1, Y, Xhalf, X_opt,
-                                 gbar_opt, 1, s);
+                                 gbar_opt, 1, live, s);
         }));
     }
     plan->stat_pending = false;

@@ -33,8 +33,10 @@ template <int B, int H, bool kBucket>
 __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const uint32_t* __restrict__ words,
                                                   int64_t worker_stride, int kc,
                                                   const float (*table)[2 * kMaxLevels],
-                                                  const float* __restrict__ bn, int64_t bn_stride)
+                                                  const float* __restrict__ bn, int64_t bn_stride, uint32_t live)
 {
+    // `live`: bit kk clear = worker kk's block is known to be all zero words, which are then not read (their
+    // symbols are 0 and add the table's +0)
     constexpr int C = B + 1;
     constexpr int kFirst = (kPartSyms * H * C) >> 5;                  // first and last word of this piece
     constexpr int kLast = ((kPartSyms * (H + 1) * C) - 1) >> 5;
@@ -43,7 +45,7 @@ __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const
     for (int kk = 0; kk < kWorkerChunk; ++kk)
 #pragma unroll
         for (int i = 0; i < C; ++i)
-            w[kk][i] = (i >= kFirst && i <= kLast && kk < kc) ? __ldcs(words + kk * worker_stride + i * 32) : 0u;
+            w[kk][i] = (i >= kFirst && i <= kLast && kk < kc && ((live >> kk) & 1u)) ? __ldcs(words + kk * worker_stride + i * 32) : 0u;
     float nr[kBucket ? kWorkerChunk : 1][kPartRows];
     if (kBucket) {
 #pragma unroll
@@ -68,6 +70,7 @@ __device__ __forceinline__ void decode_accumulate(float (&acc)[kPartSyms], const
 struct Rates { float eta, gamma, eta_cur; };
 
 struct DecodeArgs {
+    const uint32_t* live;    // per block of 1024 coordinates: bit k set = worker k's words are not all zero; or nullptr
     const uint32_t* packed;
     const float* norms;
     const float* levels;
@@ -102,7 +105,7 @@ template <int B, int H, int kMode, bool kBucket>
 __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L, int layer, const DecodeArgs& a,
                                             float (*table)[2 * kMaxLevels], const Rates& rt, float invK,
                                             int64_t blk, bool active, bool& resident, float4* stage,
-                                            double& lam_acc, double& mu_acc)
+                                            double& lam_acc, double& mu_acc, uint32_t block_live)
 {
     constexpr bool kQoda = kMode >= 1, kAlt = kMode == 2;
     const float eta = rt.eta, gamma = rt.gamma;
@@ -128,14 +131,17 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     float acc[kPartSyms];
 #pragma unroll
     for (int i = 0; i < kPartSyms; ++i) acc[i] = 0.0f;
+    uint32_t any_live = 0;
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
         const int kc = min(kWorkerChunk, K - k0);
+        const uint32_t live = block_live >> k0;          // the chunk's workers in the low bits
+        any_live |= live & ((1u << kc) - 1u);
         if (!resident) fill_tables<kBucket>(p, L, layer, a, table, k0, kc);
         if (kBucket || K <= kWorkerChunk) resident = true;
         const int64_t bn_stride = p.total_blocks * 8;
         const float* bn = kBucket ? a.norms + (int64_t)k0 * bn_stride + (L.block_off + blk) * 8 + kPartRows * H : nullptr;
         if (active) decode_accumulate<B, H, kBucket>(acc, a.packed + (int64_t)k0 * p.packed_words + woff, p.packed_words,
-                                                     kc, table, bn, bn_stride);
+                                                     kc, table, bn, bn_stride, live);
     }
     if (!active) return;
     if (kQoda) cp_async_wait<0>();
@@ -174,7 +180,7 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
                     }
                 }
             }
-            *reinterpret_cast<float4*>(a.Y + pos) = y;
+            if (any_live) *reinterpret_cast<float4*>(a.Y + pos) = y;     // no worker sent anything here: y = y0 - 0
             *reinterpret_cast<float4*>(a.Xhalf + pos) = h;
             if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
         }
@@ -197,11 +203,13 @@ __device__ __forceinline__ void decode_block_chunked(const PlanDev& p, const Lay
     for (int b0 = 0; b0 < tile.nblocks; b0 += kWarps) {
         const bool active = b0 + warp < tile.nblocks;
         const int64_t blk = tile.block0 + b0 + warp;
-        decode_half<B, 0, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
-        decode_half<B, 1, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+        // which workers sent anything in this block (all of them when that is not known)
+        const uint32_t block_live = (!kBucket && a.live && active) ? __ldg(a.live + L.block_off + blk) : 0xffffffffu;
+        decode_half<B, 0, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc, block_live);
+        decode_half<B, 1, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc, block_live);
         if (kParts == 4) {
-            decode_half<B, 2 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
-            decode_half<B, 3 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc);
+            decode_half<B, 2 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc, block_live);
+            decode_half<B, 3 % kParts, kMode, kBucket>(p, L, layer, a, table, rt, invK, blk, active, resident, stage, lam_acc, mu_acc, block_live);
         }
     }
 }
@@ -328,10 +336,10 @@ cudaError_t launch_average(const PlanDev& p, const float* Xhalf, double* xsum, c
 
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
-                          float* gbar, int mode, cudaStream_t s)
+                          float* gbar, int mode, const uint32_t* live, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
-    DecodeArgs a{packed, norms, levels, X1, Y, Xhalf, X, gbar};
+    DecodeArgs a{live, packed, norms, levels, X1, Y, Xhalf, X, gbar};
     const unsigned grid = (unsigned)p.num_tiles * p.sub_tiles;
     if (p.bucket_norm) {
         if (mode == 2)      decode_kernel<2, true><<<grid, kThreads, kStageBytes, s>>>(p, a);
@@ -342,6 +350,23 @@ cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float*
         else if (mode == 1) decode_kernel<1, false><<<grid, kThreads, kStageBytes, s>>>(p, a);
         else                decode_kernel<0, false><<<grid, kThreads, kStageBytes, s>>>(p, a);
     }
+    return cudaGetLastError();
+}
+
+// block_live[b] = bitmask of the workers whose block b holds a nonzero value, from the K zero-row mask arrays
+__global__ void __launch_bounds__(256) block_live_kernel(PlanDev p)
+{
+    const int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (b >= p.total_blocks) return;
+    uint32_t m = 0;
+    for (int k = 0; k < p.num_workers; ++k) m |= (p.row_mask[(int64_t)k * p.total_blocks + b] != 0 ? 1u : 0u) << k;
+    p.block_live[b] = m;
+}
+
+cudaError_t launch_block_live(const PlanDev& p, cudaStream_t s)
+{
+    if (p.total_blocks == 0) return cudaSuccess;
+    block_live_kernel<<<(unsigned)((p.total_blocks + 255) / 256), 256, 0, s>>>(p);
     return cudaGetLastError();
 }
 

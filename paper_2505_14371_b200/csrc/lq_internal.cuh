@@ -81,6 +81,7 @@ struct PlanDev {
     uint8_t* row_mask;    // [K][total_blocks]  bit j of a block's byte: row j (128 values) holds a nonzero value
     const uint8_t* row_mask_prev;   // the same for the input behind the previous message, or NULL when unknown
     int64_t total_blocks; // blocks of 1024 values per worker, all layers
+    uint32_t* block_live; // [total_blocks]  bit k: worker k's block holds a nonzero value (built from row_mask; K <= 32)
     double* energy_partial;   // [K][num_tiles]  bucket scope: per-tile sums of squared bucket norms
     uint32_t* flag_partial;   // [K][num_tiles]  bucket scope: bit 0 a non-finite bucket, bit 1 a nonzero bucket
     float* layer_weight;      // [K][L]          bucket scope: sqrt of a layer's summed squared bucket norms
@@ -113,9 +114,10 @@ cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint3
 cudaError_t launch_bucket_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_stat_finalize(const PlanDev& p, cudaStream_t s);
 // mode 0: decode + aggregate only; 1: + QODA update, Eq. (general_stepsize); 2: + QODA update, Eq. (Alt)
+// live: per block the bitmask of workers whose words are not all zero, for exactly this message, or nullptr
 cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float* norms,
                           const float* levels, const float* X1, float* Y, float* Xhalf, float* X,
-                          float* gbar, int mode, cudaStream_t s);
+                          float* gbar, int mode, const uint32_t* live, cudaStream_t s);
 cudaError_t launch_level_probabilities(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
                                        const float* levels, double* probs, cudaStream_t s);
 cudaError_t launch_symbol_counts(const PlanDev& p, const uint32_t* packed, uint32_t* counts, cudaStream_t s);
@@ -127,6 +129,7 @@ cudaError_t launch_entropy_encode(const PlanDev& p, const uint32_t* packed, cons
                                   uint32_t* offsets, uint32_t* out, int64_t capacity, cudaStream_t s);
 cudaError_t launch_entropy_decode(const PlanDev& p, const uint32_t* in, int64_t capacity, const uint32_t* offsets,
                                   const uint16_t* dec_tables, uint32_t* packed, uint32_t* bad, cudaStream_t s);
+cudaError_t launch_block_live(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s);
 cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_qoda_scalars(const PlanDev& p, cudaStream_t s);
