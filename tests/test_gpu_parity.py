@@ -444,3 +444,35 @@ def test_fit_levels_shared_by_type(lqm, orc):
     assert compare_messages(orc, plan, packed, ref) == (0, 0)
     with pytest.raises(lqm.LqError):
         plan.lq_fit_levels_shared(hist, norms, K, [1, 1, 1, 1, 1, 1])
+
+
+def test_update_with_and_without_the_zero_block_masks_agree():
+    """qoda_step on the buffer the encoder wrote (all-zero blocks are skipped from the masks) against qoda_step on a
+    copy of the message at another address (everything is read): identical iterates, also where no worker sent
+    anything."""
+    import paper_2505_14371_b200 as lqm
+    lqm.load_library()
+    sizes, K = [70000, 3000, 9000], 5
+    outs = []
+    for use_copy in (False, True):
+        plan = lqm.Plan(sizes, [4, 2, 6], 2, K, 5)
+        g = torch.Generator(device="cuda").manual_seed(8)
+        X1 = torch.randn(plan.padded_elems, generator=g, device="cuda")
+        Y = torch.empty_like(X1); Xh = torch.empty_like(X1); X = torch.zeros_like(X1); gbar = torch.zeros_like(X1)
+        plan.qoda_init(X1, Y, Xh)
+        pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+        for t in (1, 2, 3):
+            grads = torch.randn((K, plan.padded_elems), generator=g, device="cuda")
+            grads[:, 2048:30000] = 0.0                      # blocks that are zero for every worker
+            grads[1:, 30000:50000] = 0.0                    # blocks that only worker 0 fills
+            grads[2, :] = 0.0                               # a worker that sends nothing at all
+            c, p = t % 2, (t + 1) % 2
+            plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=pk[p] if t > 1 else None,
+                                  prev_norms=nm[p] if t > 1 else None)
+            msg = pk[c].clone() if use_copy else pk[c]
+            plan.qoda_step(msg, nm[c], X1, Y, Xh, X, gbar)
+        torch.cuda.synchronize()
+        outs.append([x.cpu().numpy().copy() for x in (Y, Xh, X, gbar)])
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+    assert not outs[0][3][2048:30000].any()                 # gbar is zero where nobody sent anything
