@@ -284,7 +284,7 @@ def run_gpu(args) -> None:
     prof = plan.lq_profile_read()
     plan.lq_profile_enable(False)
     ms = aggregate_over_ranks(local_ms, world, dev)
-    graph_ms = None
+    graph_ms, graph_error = None, None
     if args.graph and ex is None:
         # two iterations recorded once (messages and masks are double-buffered), replayed steps / 2 times; the step
         # index comes from the plan's device-side counter, so nothing in the recording changes between replays
@@ -293,20 +293,27 @@ def run_gpu(args) -> None:
             c, p = state["t"] % 2, (state["t"] + 1) % 2
             plan.lq_quantize_pack(grads, pkg.STEP_AUTO, packed[c], norms[c], prev_packed=packed[p], prev_norms=norms[p])
             plan.qoda_step(packed[c], norms[c], X1, Y, Xh)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            auto_step(); auto_step()
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        reps = max(1, args.steps // 2)
-        e0.record()
-        for _ in range(reps):
-            graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        graph_ms = aggregate_over_ranks(e0.elapsed_time(e1) / (2 * reps), world, dev)
+        try:
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                auto_step(); auto_step()
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            reps = max(1, args.steps // 2)
+            e0.record()
+            for _ in range(reps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            graph_ms = e0.elapsed_time(e1) / (2 * reps)
+        except RuntimeError as exc:      # the headline number above does not depend on this extra measurement
+            graph_error = str(exc)[:200]
+        # every rank takes part in the reduction, also one whose recording failed
+        graph_ms = aggregate_over_ranks(graph_ms if graph_ms is not None else float("inf"), world, dev)
+        if graph_ms == float("inf"):
+            graph_ms, graph_error = None, graph_error or "the recording failed on another rank"
 
     # ---- end to end: pinned host gradients in, new iterate out ------------------------------
     e2e = None
@@ -413,6 +420,8 @@ def run_gpu(args) -> None:
                        "multi_gpu": "K workers shared out over the ranks, messages by all-gather" if args.exchange
                                     else "replicas only"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "calls": calls}
+    if graph_error is not None:
+        line["cuda_graph"] = {"error": graph_error}
     if graph_ms is not None:
         line["cuda_graph"] = {"ms_per_step": graph_ms, "value": whole_job_value(4.0 * K * D * share / 1e9, world, graph_ms),
                               "note": "the same two calls per step, two steps recorded once and replayed"}
