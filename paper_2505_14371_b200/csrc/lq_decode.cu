@@ -131,11 +131,9 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     float acc[kPartSyms];
 #pragma unroll
     for (int i = 0; i < kPartSyms; ++i) acc[i] = 0.0f;
-    uint32_t any_live = 0;
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
         const int kc = min(kWorkerChunk, K - k0);
         const uint32_t live = block_live >> k0;          // the chunk's workers in the low bits
-        any_live |= live & ((1u << kc) - 1u);
         if (!resident) fill_tables<kBucket>(p, L, layer, a, table, k0, kc);
         if (kBucket || K <= kWorkerChunk) resident = true;
         const int64_t bn_stride = p.total_blocks * 8;
@@ -180,7 +178,7 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
                     }
                 }
             }
-            if (any_live) *reinterpret_cast<float4*>(a.Y + pos) = y;     // no worker sent anything here: y = y0 - 0
+            if (block_live) *reinterpret_cast<float4*>(a.Y + pos) = y;   // no worker sent anything here: y = y0 - 0
             *reinterpret_cast<float4*>(a.Xhalf + pos) = h;
             if (a.X) *reinterpret_cast<float4*>(a.X + pos) = x;
         }
