@@ -58,6 +58,9 @@ def test_random_plan_against_the_oracle(orc, case):
     plan.qoda_init(X1, Y, Xh); model.qoda_init(to_unpadded(plan, X1))
     pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
     off = plan.elem_offsets
+    # fp64 sums of up to D * K non-negative terms in two different orders: the oracle adds them one after the other,
+    # which can lose up to one rounding of the running total per term
+    sum_tol = max(1e-12, 2.0 * K * sum(sizes) * 2.0 ** -53)
     for t in range(1, 6):
         if rng.random() < 0.4:                                   # new level tables for some layers
             for m in range(L):
@@ -94,16 +97,16 @@ def test_random_plan_against_the_oracle(orc, case):
             assert np.array_equal(hist.cpu().numpy().view(np.uint32)[:, :L], ref["hist"]), tag
         if alt == 0.0:
             sq, _ = plan.lq_get_statistics()
-            assert _close(sq.numpy(), ref["sq_diff"], 1e-12), tag
+            assert _close(sq.numpy(), ref["sq_diff"], sum_tol), tag
         gref = model.qoda_step()
         assert np.array_equal(to_unpadded(plan, gbar), gref), tag
         tt, S, eta = plan.qoda_get_scalars()
         assert tt == t + 1 and eta == float(model.eta), tag
         if alt:
             lam, mu, gamma = plan.qoda_get_alt_scalars()
-            assert gamma == float(model.gamma) and abs(lam - model.lam) <= 1e-12 * max(model.lam, 1e-300), tag
+            assert gamma == float(model.gamma) and abs(lam - model.lam) <= sum_tol * max(model.lam, 1e-300), tag
         else:
-            assert abs(S - model.S) <= 1e-12 * max(model.S, 1e-300), tag
+            assert abs(S - model.S) <= sum_tol * max(model.S, 1e-300), tag
         for got, want in [(Y, model.Y), (Xh, model.Xhalf), (X, model.X)]:
             assert _close(to_unpadded(plan, got), want, 1e-6), tag
         assert _close(to_unpadded(plan, xsum), model.xsum, 1e-6), tag      # running sum of X_{s+1/2}, s <= t
