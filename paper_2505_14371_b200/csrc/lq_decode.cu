@@ -133,7 +133,9 @@ __device__ __forceinline__ void decode_half(const PlanDev& p, const LayerDesc& L
     for (int i = 0; i < kPartSyms; ++i) acc[i] = 0.0f;
     for (int k0 = 0; k0 < K; k0 += kWorkerChunk) {
         const int kc = min(kWorkerChunk, K - k0);
-        const uint32_t live = block_live >> k0;          // the chunk's workers in the low bits
+        // the chunk's workers in the low bits; the masks cover at most 32 workers, and beyond that (masks unknown,
+        // block_live all ones) every word is read: a shift by 32 or more is not defined
+        const uint32_t live = k0 < 32 ? block_live >> k0 : 0xffffffffu;
         if (!resident) fill_tables<kBucket>(p, L, layer, a, table, k0, kc);
         if (kBucket || K <= kWorkerChunk) resident = true;
         const int64_t bn_stride = p.total_blocks * 8;

@@ -169,7 +169,7 @@ def test_zero_rows_and_negative_zero(lqm, orc):
         assert _close(sq.numpy(), ref["sq_diff"], 1e-12), step
 
 
-@pytest.mark.parametrize("K", [1, 4, 11, 16])
+@pytest.mark.parametrize("K", [1, 4, 11, 16, 33, 40])
 def test_decode_aggregate_worker_counts(lqm, orc, K):
     sizes = [4100, 7, 1024, 2049]
     plan = lqm.Plan(sizes, [4, 8, 1, 3], 0, K, SEED)
@@ -262,6 +262,30 @@ def test_qoda_multi_step_small(lqm, orc):
         model.qoda_step()
         tt, S, eta = plan.qoda_get_scalars()
         assert tt == t + 1 and abs(S - model.S) <= 1e-12 * model.S and eta == float(model.eta)
+        assert _close(to_unpadded(plan, Y), model.Y, 1e-6) and _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
+
+
+def test_qoda_step_more_than_32_workers(lqm, orc):
+    """K = 37: the decoder's per-block worker bitmask covers 32 workers, so every word must be read; three
+    iterations of encode + fused update against the oracle, with blocks that only some workers fill."""
+    sizes, K = [5000, 33, 2048], 37
+    plan = lqm.Plan(sizes, [3, 5, 4], 2, K, SEED)
+    model = oracle_model(orc, plan)
+    X1 = _grads(plan, 5)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    model.qoda_init(to_unpadded(plan, X1))
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    for t in range(1, 4):
+        grads = _grads(plan, 2000 + t)
+        grads[:30, 1024:3072] = 0.0                     # blocks that only workers 30..36 fill
+        grads[34:, :1024] = 0.0
+        c, p = t % 2, (t + 1) % 2
+        plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=None if t == 1 else pk[p],
+                              prev_norms=None if t == 1 else nm[p])
+        plan.qoda_step(pk[c], nm[c], X1, Y, Xh)
+        ref = model.quantize(to_unpadded(plan, grads), t)
+        assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+        model.qoda_step()
         assert _close(to_unpadded(plan, Y), model.Y, 1e-6) and _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
 
 
