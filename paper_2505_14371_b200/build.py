@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "liblq.so")
 # (source, extra flags).  The level fit is compiled without FMA contraction.
-SOURCES = [("lq_api.cu", []), ("lq_norm.cu", []), ("lq_quantize.cu", []), ("lq_decode.cu", []), ("lq_noalloc.cu", []), ("lq_coding.cu", []),
+SOURCES = [("lq_api.cu", []), ("lq_norm.cu", []), ("lq_quantize.cu", []), ("lq_quantize_bucket.cu", []), ("lq_decode.cu", []), ("lq_noalloc.cu", []), ("lq_coding.cu", []),
            ("lq_fit.cu", ["-fmad=false"]), ("lq_codelen.cu", ["-fmad=false"])]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

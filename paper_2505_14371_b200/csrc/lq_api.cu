@@ -70,6 +70,7 @@ struct lq_plan {
     uint64_t seed = 0;
     LayerDesc* d_layers = nullptr;
     Tile* d_tiles = nullptr;
+    int32_t* d_tile_order = nullptr;
     float* d_levels_stage = nullptr;
     float* d_levels_enc[2] = {nullptr, nullptr};
     SearchTables search{};         // derived from d_levels_enc[cur]
@@ -103,9 +104,9 @@ namespace {
 void free_plan(lq_plan* p)
 {
     if (!p) return;
-    cudaFree(p->d_layers); cudaFree(p->d_tiles);
+    cudaFree(p->d_layers); cudaFree(p->d_tiles); cudaFree(p->d_tile_order);
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
-    cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
+    cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast); cudaFree(p->search.first);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
     cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     cudaFree(p->dev.block_live);
@@ -249,13 +250,33 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     const size_t lev = (size_t)(num_layers ? num_layers : 1) * kLevelStride;
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_layers, p->layers.size());
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_tiles, p->tiles.size());
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_tile_order, p->tiles.size());
+    if (e == cudaSuccess && !p->tiles.empty()) {
+        // the encoder's launch order: tiles sorted by their relative position inside their layer, so that every
+        // layer is under way from the first wave of CTAs to the last
+        std::vector<int32_t> order;
+        try { order.resize(p->tiles.size()); } catch (const std::bad_alloc&) { free_plan(p); return fail(LQ_ENOMEM, "host allocation failed"); }
+        for (size_t i = 0; i < order.size(); ++i) order[i] = (int32_t)i;
+        const std::vector<LayerDesc>& Ls = p->layers;
+        const std::vector<Tile>& Ts = p->tiles;
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+            const LayerDesc& La = Ls[(size_t)Ts[(size_t)a].layer];
+            const LayerDesc& Lb = Ls[(size_t)Ts[(size_t)b].layer];
+            // (2 i + 1) / (2 n) compared exactly by cross-multiplication
+            const int64_t ka = (2 * (int64_t)(a - La.first_tile) + 1) * Lb.ntiles;
+            const int64_t kb = (2 * (int64_t)(b - Lb.first_tile) + 1) * La.ntiles;
+            return ka != kb ? ka < kb : a < b;
+        });
+        e = cudaMemcpy(p->d_tile_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    }
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_stage, lev);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[0], lev);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[1], lev);
     const size_t nl = (size_t)(num_layers ? num_layers : 1);
-    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.lut, nl * kLutStride);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.lut, nl * kLutEntries);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.ld, nl * kMaxLevels);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.fast, nl);
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.first, nl);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT * (size_t)d.sub_tiles);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.stat_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
@@ -298,7 +319,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
         free_plan(p);
         return fail(code, "plan setup: %s", cudaGetErrorString(e));
     }
-    d.layers = p->d_layers; d.tiles = p->d_tiles;
+    d.layers = p->d_layers; d.tiles = p->d_tiles; d.tile_order = p->d_tile_order;
     e = launch_build_search(d, p->d_levels_enc[0], p->search, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -424,8 +445,9 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_PARTIAL, s, [&] { return launch_norm_partial(d, grads, true, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_NORM_FINALIZE, s, [&] { return launch_norm_finalize(d, norms, s); }));
     LQ_CUDA(timed(plan, LQ_KERNEL_QUANTIZE_PACK, s, [&] {
+        // under Eq. (Alt) nothing consumes the statistic of Eq. (general_stepsize): it is left out (and reads 0)
         return launch_quantize(d, grads, step, packed, norms, hist, prev_packed, prev_norms, lc, lp,
-                               plan->search, s);
+                               plan->search, plan->alt_qhat <= 0.0, s);
     }));
     LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_stat_finalize(d, s); }));
     plan->have_message = true;

@@ -17,8 +17,8 @@ constexpr int kThreads = 256;
 constexpr int kLevelStride = 256;     // floats per layer in a level table
 constexpr int kMaxLevels = 256;
 constexpr int kCodeMaxLen = 12;       // longest code word of the entropy stage (LQ_CODE_MAX_LEN)
-constexpr int kLutStride = 392;       // uint2 entries per layer in the search table (386 used)
-constexpr uint32_t kLutClamp = 0x33780000u;   // bit pattern one histogram bin below 2^-24
+constexpr int kLutEntries = 2048;     // u32 entries per layer in the encoder's search table: one per value of the
+                                      // top 13 bits of a non-negative float (16 bins per octave); 2033 are reachable
 
 struct LayerDesc {
     int64_t elem_off;     // first element of the layer inside a worker's fp32 row
@@ -56,6 +56,8 @@ struct QodaScalars {
 struct PlanDev {
     const LayerDesc* layers;
     const Tile* tiles;
+    const int32_t* tile_order;   // the order in which the encoder's CTAs take the tiles: all layers advance together, so
+                                 // that layers of different character (dense, mostly zero rows) share the SMs at any time
     int32_t num_layers;
     int32_t num_tiles;
     int32_t num_workers;
@@ -97,15 +99,16 @@ cudaError_t launch_norm_partial(const PlanDev& p, const float* grads, bool write
 cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s);
 // Encode-side tables derived from one level table (rebuilt whenever the levels change).
 struct SearchTables {
-    uint2* lut;        // [L][kLutStride]  {8 * tau0, bits of the level inside the bin or +inf}
+    uint32_t* lut;     // [L][kLutEntries] per bin: 8 * tau0 | (low 19 bits of the level inside the bin, minus 1) << 13
     float2* ld;        // [L][kMaxLevels]  {l_tau, l_{tau+1} - l_tau}
-    int32_t* fast;     // [L]              1 if every histogram bin holds at most one level
+    int32_t* fast;     // [L]              1 if every bin holds at most one level
+    int32_t* first;    // [L]              first bin whose entry differs from that of bin 0 (the bins below hold no level)
 };
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s);
 cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
                             const float* norms, uint32_t* hist, const uint32_t* prev_packed,
                             const float* prev_norms, const float* levels_cur,
-                            const float* levels_prev, SearchTables t, cudaStream_t s);
+                            const float* levels_prev, SearchTables t, bool need_stat, cudaStream_t s);
 // bucket scope: `bucket_norms` [K][8 * total_blocks] is written, `prev_norms` has the same shape
 cudaError_t launch_quantize_bucketed(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,
                                      float* bucket_norms, uint32_t* hist, const uint32_t* prev_packed,
