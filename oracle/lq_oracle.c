@@ -135,15 +135,6 @@ void orc_quantize_layer(const float* v, int64_t d, int64_t first_index, float no
     if (near) *near = near_count;
 }
 
-/* Probability of rounding up for one normalised value (xi(u), Section 3.1), in fp64. */
-double orc_round_up_probability(double u, const float* level, int n, int* tau_out)
-{
-    int tau = 0;
-    for (int j = 1; j <= n - 2; ++j) if ((double)level[j] <= u) tau = j;
-    if (tau_out) *tau_out = tau;
-    return (u - (double)level[tau]) / ((double)level[tau + 1] - (double)level[tau]);
-}
-
 /* ------------------------------------------------------------------------------------
  * Fixed-width message layout (Section 3.2: a 32-bit float norm, one sign bit and one
  * integer code per coordinate; Section 7.1 footnote: no entropy code on top).

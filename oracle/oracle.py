@@ -46,8 +46,6 @@ def lib():
         L.orc_quantize_layer.argtypes = [f32p, C.c_int64, C.c_int64, C.c_float, f32p, C.c_int, C.c_uint64,
                                          C.c_uint32, C.c_uint32, C.c_uint32, u8p, u8p,
                                          C.POINTER(C.c_int64)]
-        L.orc_round_up_probability.restype = C.c_double
-        L.orc_round_up_probability.argtypes = [C.c_double, f32p, C.c_int, C.POINTER(C.c_int)]
         L.orc_packed_words.restype = C.c_int64
         L.orc_packed_words.argtypes = [C.c_int64, C.c_int]
         L.orc_pack_layer.argtypes = [u8p, u8p, C.c_int64, C.c_int, u32p]
@@ -127,12 +125,6 @@ def quantize_layer(v, norm, levels, seed, step, worker, layer, first_index=0):
                              levels.size, seed, step, worker, layer, _p(idx, C.c_uint8),
                              _p(sg, C.c_uint8), C.byref(near))
     return idx, sg, near.value
-
-
-def round_up_probability(u: float, levels) -> tuple:
-    levels = _f32(levels); tau = C.c_int(0)
-    xi = lib().orc_round_up_probability(float(u), _p(levels, C.c_float), levels.size, C.byref(tau))
-    return float(xi), tau.value
 
 
 def packed_words(d: int, b: int) -> int:
