@@ -156,9 +156,12 @@ int lq_layer_norms(lq_plan* plan, const float* grads, float* norms, void* stream
  *     sum_k ||V^_{k,t+1/2} - V^_{k,t-1/2}||^2 of Eq. (general_stepsize), which is left
  *     inside the plan for the next qoda_step: per coordinate the fp32 difference of the two
  *     decoded fp32 values, its square summed in fp64.  The previous message is decoded with the
- *     levels it was encoded with, even if the levels were changed in between.  It MUST be the
- *     output of this plan's previous lq_quantize_pack call: the plan remembers which rows of
- *     that call's input were all zero and does not read the corresponding words again.
+ *     levels it was encoded with, even if the levels were changed in between.  It must hold the
+ *     message of this plan's previous lq_quantize_pack call (that message's levels and norms
+ *     decode it).  When it is the very buffer that call wrote, the plan uses what it remembers of
+ *     that call - which rows of its input were all zero - and does not read the corresponding
+ *     words again; a copy at another address is read in full.  A caller that rewrote the buffer
+ *     in place says so with lq_message_modified.
  *   prev_packed must not alias packed.
  *   The sign of a coordinate is (v < 0): +0 and -0 both give symbol 0, so rows of zeros (of either
  *   sign) become all-zero words; such rows are detected by the norm pass and not read again.
@@ -216,11 +219,14 @@ int qoda_init(lq_plan* plan, const float* X1, float* Y, float* Xhalf, void* stre
  * is no new one).  When `packed` is the very buffer that call wrote for all K workers (layer or global scope),
  * the buffer must still hold that message: blocks the encoder knows to be all zero are not read again, and where no
  * worker sent anything Y is left as it is.  A message at another address, and one assembled from several worker
- * ranges, is read in full.
+ * ranges, is read in full; so is that buffer after lq_message_modified, the call by which a caller who has
+ * rewritten the buffer in place (its own exchange, say) tells the plan that what it remembers of the last
+ * lq_quantize_pack's input no longer describes the words there.  The next lq_quantize_pack starts afresh.
  *   packed dev [K][W], norms dev [K][L], X1 dev [D_pad] in;  Y dev [D_pad] in/out;
  *   Xhalf dev [D_pad] out (X_{t+3/2});  X_opt, gbar_opt: NULL or dev [D_pad] out. */
 int qoda_step(lq_plan* plan, const uint32_t* packed, const float* norms, const float* X1,
               float* Y, float* Xhalf, float* X_opt, float* gbar_opt, void* stream);
+int lq_message_modified(lq_plan* plan);
 
 /* Code-length accounting (appendix on the coding framework).
  * lq_level_probabilities: for every layer, the probability p^_j that level j is emitted,
@@ -291,9 +297,14 @@ int qoda_set_average(lq_plan* plan, double* xsum, void* stream);
  *   eta_{t+1} = fp32((1 + lambda_{t-1} + mu_{t-1})^(-1/2)),  gamma_{t+1} = fp32((1 + lambda_{t-1})^(q_hat - 1/2)),
  *   lambda_t = sum_{s<=t} ||gbar_{s+1/2}||^2,  mu_t = sum_{s<=t} ||X_s - X_{s+1}||^2  (fp64 sums of squares of
  *   fp32 values; both start at 0 in qoda_init, so eta_1 = eta_2 = gamma_1 = gamma_2 = 1),
+ * where gbar is the mean of the K decoded messages: lambda is the appendix's form, the squared norm of the
+ * AGGREGATE, sum_s ||sum_k V^_{k,s+1/2}||^2 / K^2, which the proofs use.  The display of Eq. (Alt) in the main
+ * text sums the K workers' squared norms instead (sum_s sum_k ||V^_{k,s+1/2}||^2 / K^2, larger by up to a
+ * factor K); that form is not computed here.
  * X_{t+1} = fma(eta_{t+1}, Y_{t+1}, X_1), X_{t+3/2} = fma(-gamma_{t+1}, gbar, X_{t+1}), and adds this
  * iteration's terms to lambda and mu afterwards.  The statistic of lq_quantize_pack is not used, so
- * its prev_packed / prev_norms may be NULL.  q_hat = 0 switches back to Eq. (general_stepsize).
+ * its prev_packed / prev_norms may be NULL; while this schedule is on, lq_quantize_pack does not compute it
+ * either (lq_get_statistics then reads zeros), except in calls that also collect histograms.  q_hat = 0 switches back to Eq. (general_stepsize).
  * Choose the schedule before qoda_init: the two schedules keep separate sums. */
 int qoda_set_alt_rates(lq_plan* plan, double q_hat);
 /* Host copies of lambda, mu and the current gamma; synchronises.  Any output may be NULL. */

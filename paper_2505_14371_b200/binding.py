@@ -23,7 +23,7 @@ STATUS_NONFINITE = 2
 STEP_AUTO = 0xFFFFFFFF          # lq_quantize_pack: take the step index from the plan's device-side iteration counter
 
 EXPORTS = ["lq_plan_create", "lq_plan_destroy", "lq_plan_padded_elems", "lq_plan_packed_words",
-           "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_worker_range", "lq_side_data_export",
+           "lq_plan_layer_info", "lq_set_norm_scope", "lq_plan_norm_count", "lq_layer_weights", "lq_set_worker_range", "lq_message_modified", "lq_side_data_export",
            "lq_side_data_import", "lq_set_levels", "lq_get_levels", "lq_layer_norms",
            "lq_quantize_pack", "lq_fit_levels", "lq_fit_levels_shared", "lq_decode_aggregate", "qoda_init", "qoda_step",
            "qoda_get_scalars", "lq_code_build", "lq_code_universal", "lq_code_set", "lq_code_get", "lq_plan_blocks", "lq_entropy_encode",
@@ -61,6 +61,7 @@ def load_library() -> C.CDLL:
     L.lq_plan_norm_count.restype = i64
     L.lq_layer_weights.argtypes = [vp, vp]
     L.lq_set_worker_range.argtypes = [vp, i32, i32]
+    L.lq_message_modified.argtypes = [vp]
     L.lq_side_data_export.argtypes = [vp, vp, vp, vp, vp]
     L.lq_side_data_import.argtypes = [vp, vp, vp, vp, vp]
     L.lq_set_levels.argtypes = [vp, i32, C.POINTER(C.c_float), i32]
@@ -186,6 +187,9 @@ class Plan:
         """"layer" (default), "global" (one norm over the worker's whole vector) or "bucket" (one norm per 128
         consecutive coordinates of a layer; norms buffers then have lq_plan_norm_count() values per worker)."""
         _check(load_library().lq_set_norm_scope(self._h, {"layer": 0, "global": 1, "bucket": 2}[scope]))
+
+    def lq_message_modified(self) -> None:
+        _check(load_library().lq_message_modified(self._h))
 
     def lq_set_worker_range(self, first_worker: int, count: int) -> None:
         _check(load_library().lq_set_worker_range(self._h, int(first_worker), int(count)))

@@ -92,6 +92,7 @@ struct lq_plan {
     uint8_t* d_row_mask[2] = {nullptr, nullptr};   // zero-row masks of the last two encoded inputs
     int mask_cur = 0;
     bool masks_known = false;              // d_row_mask[mask_cur] describes the last message of the current worker range
+    bool message_intact = false;           // ... and the caller has not said that it rewrote that message (lq_message_modified)
     // optional per-kernel timing (lq_profile_enable): event pairs recorded around each launch
     struct ProfRec { int id; cudaEvent_t a, b; };
     bool profiling = false;
@@ -144,7 +145,7 @@ cudaError_t timed(lq_plan* p, int id, cudaStream_t s, F&& launch)
 const uint32_t* message_masks(const lq_plan* p, const uint32_t* packed)
 {
     const PlanDev& d = p->dev;
-    if (!p->have_message || !p->masks_known || d.bucket_norm || packed != p->last_packed) return nullptr;
+    if (!p->have_message || !p->masks_known || !p->message_intact || d.bucket_norm || packed != p->last_packed) return nullptr;
     if (d.worker0 != 0 || d.worker_count != d.num_workers || d.num_workers > 32) return nullptr;
     return d.block_live;
 }
@@ -425,7 +426,10 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
         plan->prev = plan->cur;
     }
     // the masks written now describe this message; the ones of the last call describe prev_packed
-    plan->dev.row_mask_prev = (plan->have_message && plan->masks_known) ? plan->d_row_mask[plan->mask_cur] : nullptr;
+    // (they describe prev_packed only if that is the very message the last call wrote, untouched since; for any
+    // other previous message every row is taken as possibly nonzero)
+    plan->dev.row_mask_prev = (plan->have_message && plan->masks_known && plan->message_intact && prev_packed == plan->last_packed)
+                                  ? plan->d_row_mask[plan->mask_cur] : nullptr;
     plan->mask_cur = plan->have_message ? 1 - plan->mask_cur : plan->mask_cur;
     plan->dev.row_mask = plan->d_row_mask[plan->mask_cur];
     const PlanDev& d = plan->dev;
@@ -439,6 +443,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
         LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_bucket_finalize(d, s); }));
         plan->have_message = true;
         plan->masks_known = true;          // (no masks in this scope: the flag also marks an unbroken stream of messages)
+        plan->message_intact = true;
         plan->stat_pending = true;
         return LQ_OK;
     }
@@ -452,6 +457,7 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
     LQ_CUDA(timed(plan, LQ_KERNEL_STAT_FINALIZE, s, [&] { return launch_stat_finalize(d, s); }));
     plan->have_message = true;
     plan->masks_known = true;
+    plan->message_intact = true;
     plan->last_packed = packed;
     plan->stat_pending = true;
     return LQ_OK;
@@ -595,6 +601,13 @@ int lq_set_norm_scope(lq_plan* plan, int32_t scope)
         return fail(LQ_ESTATE, "the bucket scope can only be entered or left before the first lq_quantize_pack");
     plan->dev.global_norm = scope == LQ_NORM_GLOBAL ? 1 : 0;
     plan->dev.bucket_norm = bucket;
+    return LQ_OK;
+}
+
+int lq_message_modified(lq_plan* plan)
+{
+    if (!plan) return fail(LQ_EINVAL, "plan is NULL");
+    plan->message_intact = false;
     return LQ_OK;
 }
 

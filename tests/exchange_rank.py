@@ -37,7 +37,8 @@ def run(rank: int, world: int, scope: str, group_ready: bool):
     tt, S, eta = plan.qoda_get_scalars()
     return dict(Y=Y.cpu().numpy(), Xh=Xh.cpu().numpy(), X=X.cpu().numpy(), gbar=gbar.cpu().numpy(),
                 packed=ex.packed[ex.cur].cpu().numpy(), norms=ex.norms[ex.cur].cpu().numpy(),
-                scalars=np.array([tt, S, eta]), levels=np.array(plan.lq_get_levels(0), np.float32))
+                scalars=np.array([tt, S, eta]), levels=np.array(plan.lq_get_levels(0), np.float32),
+                **{f"levels{m}": np.array(plan.lq_get_levels(m), np.float32) for m in range(len(SIZES))})
 
 
 if __name__ == "__main__":

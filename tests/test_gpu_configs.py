@@ -7,6 +7,7 @@ rounding threshold (fewer than 1e-6 of all coordinates), norms relative 1e-6, de
 values relative 1e-6, QODA iterates relative 1e-5.
 """
 import math
+import os
 
 import numpy as np
 import pytest
@@ -219,6 +220,18 @@ def test_config4_transformer_xl_full_size_sampled(lqm, orc):
         ref, st = orc.layer_norm(v, w.q)
         assert st == 0 and abs(float(norms[k, m]) - float(ref)) <= 1e-6 * float(ref), (k, m)
 
+    # the oracle's own norm of every (worker, layer) whose blocks are sampled below: the GPU's must equal it, and
+    # the oracle quantizes with its own (the input is the same in both iterations, hence so is the norm)
+    oracle_norms = {}
+
+    def oracle_norm(k, m):
+        if (k, m) not in oracle_norms:
+            v = grads[k, plan.elem_offsets[m]: plan.elem_offsets[m] + w.layer_sizes[m]].cpu().numpy()
+            ref, st = orc.layer_norm(v, w.q)
+            assert st == 0 and norms[k, m] == ref and norms_prev[k, m] == ref, (k, m)
+            oracle_norms[(k, m)] = ref
+        return oracle_norms[(k, m)]
+
     # sampled blocks: symbols of every worker, then the aggregate and the update, one block range at a time
     def check_blocks(m, b0, nb):
         d = w.layer_sizes[m]
@@ -227,14 +240,15 @@ def test_config4_transformer_xl_full_size_sampled(lqm, orc):
         decoded = np.zeros((K, hi - lo), np.float32); sq_part = np.zeros(K)
         for k in range(K):
             v = grads[k, e0 + lo: e0 + hi].cpu().numpy()
-            idx, sg, _ = orc.quantize_layer(v, norms[k, m], levels[m], W.PHILOX_SEED, 2, k, m, first_index=lo)
+            on = oracle_norm(k, m)
+            idx, sg, _ = orc.quantize_layer(v, on, levels[m], W.PHILOX_SEED, 2, k, m, first_index=lo)
             wo = plan.word_offsets[m] + b0 * 32 * C
             words = pk[0][k, wo: wo + nb * 32 * C].cpu().numpy().view(np.uint32)
             gi, gs = orc.unpack_layer(words, hi - lo, w.bits)
             assert np.array_equal(gi, idx) and np.array_equal(gs, sg), (m, b0, k)
-            decoded[k] = orc.decode_layer(idx, sg, norms[k, m], levels[m])
-            pidx, psg, _ = orc.quantize_layer(v, norms_prev[k, m], uniform, W.PHILOX_SEED, 1, k, m, first_index=lo)
-            sq_part[k] = orc.sq_diff(decoded[k], orc.decode_layer(pidx, psg, norms_prev[k, m], uniform))
+            decoded[k] = orc.decode_layer(idx, sg, on, levels[m])
+            pidx, psg, _ = orc.quantize_layer(v, on, uniform, W.PHILOX_SEED, 1, k, m, first_index=lo)
+            sq_part[k] = orc.sq_diff(decoded[k], orc.decode_layer(pidx, psg, on, uniform))
         want = orc.aggregate(decoded)
         assert np.array_equal(gbar[e0 + lo: e0 + hi].cpu().numpy(), want), (m, b0)
         y = Y_before[e0 + lo: e0 + hi].cpu().numpy().copy(); x1 = X1[e0 + lo: e0 + hi].cpu().numpy()
@@ -263,6 +277,62 @@ def test_config4_transformer_xl_full_size_sampled(lqm, orc):
     assert torch.equal(Y[emb][zero_all], Y_before[emb][zero_all]) and bool((gbar[emb][zero_all] == 0).all())
     assert bool(torch.isfinite(Xh).all()) and bool(torch.isfinite(Y).all())
     assert abs(eta - 1.0 / math.sqrt(1.0 + S)) <= 1e-6 * eta
+
+
+def test_config4_transformer_xl_two_whole_workers(lqm, orc):
+    """The same two iterations with the oracle run over two WHOLE workers of the full-size workload (the K workers'
+    layers dealt to host threads; the C routines release the interpreter lock): every layer's norm, every word of
+    their messages and every layer's term of the step-size statistic; then S and eta from the GPU's own terms."""
+    from concurrent.futures import ThreadPoolExecutor
+    from paper_2505_14371_b200 import workloads as W
+    if torch.cuda.mem_get_info()[0] < 20e9:
+        pytest.skip("needs about 12 GB of free device memory")
+    w = W.transformer_xl_workload()
+    K, Lr = w.num_workers, w.num_layers
+    plan = lqm.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, "cuda")
+    pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+    X1 = torch.zeros(plan.padded_elems, device="cuda"); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+    plan.qoda_init(X1, Y, Xh)
+    hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, pk[1], nm[1], hist=hist)
+    plan.lq_fit_levels(hist, nm[1], K)
+    plan.qoda_step(pk[1], nm[1], X1, Y, Xh)
+    _, S1, _ = plan.qoda_get_scalars()
+    plan.lq_quantize_pack(grads, 2, pk[0], nm[0], prev_packed=pk[1], prev_norms=nm[1])
+    plan.qoda_step(pk[0], nm[0], X1, Y, Xh)
+    torch.cuda.synchronize()
+    _, S2, eta = plan.qoda_get_scalars()
+    sq, _ = plan.lq_get_statistics()
+    levels = [np.array(plan.lq_get_levels(m), np.float32) for m in range(Lr)]
+    uniform = orc.uniform_levels(w.bits)
+    norms = nm[0].cpu().numpy()
+    workers = (0, 5)
+    host = {k: grads[k].cpu().numpy() for k in workers}
+    words = {k: pk[0][k].cpu().numpy().view(np.uint32) for k in workers}
+
+    def one_layer(job):
+        k, m = job
+        d = w.layer_sizes[m]
+        v = host[k][plan.elem_offsets[m]: plan.elem_offsets[m] + d]
+        on, st = orc.layer_norm(v, w.q)
+        idx, sg, _ = orc.quantize_layer(v, on, levels[m], W.PHILOX_SEED, 2, k, m)
+        got = words[k][plan.word_offsets[m]: plan.word_offsets[m] + orc.packed_words(d, w.bits)]
+        same = bool(np.array_equal(got, orc.pack_layer(idx, sg, w.bits)))
+        pidx, psg, _ = orc.quantize_layer(v, on, uniform, W.PHILOX_SEED, 1, k, m)
+        term = orc.sq_diff(orc.decode_layer(idx, sg, on, levels[m]), orc.decode_layer(pidx, psg, on, uniform))
+        return k, m, st, on, same, term
+
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+        results = list(pool.map(one_layer, [(k, m) for k in workers for m in range(Lr)]))
+    for k, m, st, on, same, term in results:
+        assert st == 0 and norms[k, m] == on, (k, m)
+        assert same, (k, m)
+        assert abs(float(sq[k, m]) - term) <= max(1e-12, 2.0 * w.layer_sizes[m] * 2.0 ** -53) * term, (k, m)
+    # the running sum and the step size follow from the terms the GPU reports for all K workers
+    delta = float(sq.numpy().astype(np.float64).sum()) / (K * K)
+    assert abs((S2 - S1) - delta) <= 1e-12 * delta
+    assert abs(eta - 1.0 / math.sqrt(1.0 + S2)) <= 1e-6 * eta
 
 
 def test_config4_bucket_scope_full_size_sampled(lqm, orc):

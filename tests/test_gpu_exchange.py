@@ -40,6 +40,55 @@ def test_two_ranks_equal_one_process(tmp_path, scope):
         got = np.load(tmp_path / f"rank{r}.npz")
         for key in want:
             assert np.array_equal(got[key], want[key]), (r, key)
+    _check_against_oracle(dict(np.load(tmp_path / "rank0.npz")), scope)
+
+
+def _check_against_oracle(got, scope):
+    """Rank 0's final state against the CPU oracle run over the same three iterations (the fitted levels are taken
+    from the GPU, as in the other parity tests: the level fit has its own test)."""
+    import torch
+    import exchange_rank as R
+    import paper_2505_14371_b200 as lqm
+    from oracle import oracle as orc
+    from helpers import to_unpadded, bucket_norms_by_layer
+    orc.build()
+    plan = lqm.Plan(R.SIZES, R.BITS, R.Q, R.K, R.SEED)              # only for the padded layout
+    plan.lq_set_norm_scope(scope)
+    model = orc.OracleModel(R.SIZES, R.BITS, R.Q, R.K, R.SEED)
+    model.norm_scope = scope
+    g = torch.Generator(device="cuda").manual_seed(5)
+    X1 = torch.randn(plan.padded_elems, generator=g, device="cuda") * 0.1
+    model.qoda_init(to_unpadded(plan, X1))
+    ref = None
+    for t in (1, 2, 3):
+        grads = torch.randn((R.K, plan.padded_elems), generator=g, device="cuda") * (0.5 ** t)
+        grads[1, 100:700] = 0.0
+        ref = model.quantize(to_unpadded(plan, grads), t)
+        model.qoda_step()
+        if t == 1:
+            for m in range(len(R.SIZES)):
+                model.levels[m] = got[f"levels{m}"]
+    packed = got["packed"].view(np.uint32)
+    for k in range(R.K):
+        for m, (d, b) in enumerate(zip(R.SIZES, R.BITS)):
+            words = packed[k, plan.word_offsets[m]: plan.word_offsets[m] + orc.packed_words(d, b)]
+            assert np.array_equal(words, ref["packed"][k][m]), (k, m)
+    if scope == "layer":
+        assert np.array_equal(got["norms"][:, :len(R.SIZES)], ref["norms"])
+    else:
+        by_layer, stray = bucket_norms_by_layer(plan, torch.from_numpy(got["norms"]))
+        assert stray == 0.0
+        for m in range(len(R.SIZES)):
+            for k in range(R.K):
+                assert np.array_equal(by_layer[m][k], ref["bucket_norms"][k][m]), (k, m)
+    tt, S, eta = got["scalars"]
+    assert tt == 4 and abs(S - model.S) <= 1e-12 * model.S and eta == float(model.eta)
+
+    def unpad(a):
+        return np.concatenate([a[o:o + d] for o, d in zip(plan.elem_offsets, R.SIZES)])
+    for key, want in (("Y", model.Y), ("Xh", model.Xhalf), ("X", model.X)):
+        a = unpad(got[key])
+        assert np.max(np.abs(a - want)) <= 1e-6 * np.max(np.abs(want)), key
 
 
 def test_changing_the_range_restarts_the_message_stream():

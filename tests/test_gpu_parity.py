@@ -242,6 +242,95 @@ def test_fit_levels_parity(lqm, orc):
     assert _close(sq.numpy(), ref2["sq_diff"], 1e-12)
 
 
+def test_fitted_levels_minimise_the_variance_on_the_samples(lqm):
+    """The GPU's fitted levels checked against the paper's objective directly, without the oracle's solver: the
+    weighted variance per unit norm (Eq. Var with the weights of Eq. cdf_weight), evaluated on the samples in numpy,
+    is smaller at the fitted levels than at perturbed, uniform or exponential levels, and every interior level
+    satisfies the first-order condition int_a^b (u - a) dF~ = int_b^c (c - u) dF~ on the samples."""
+    K, d = 3, 300000
+    rng = np.random.default_rng(2024)
+    plan = lqm.Plan([d, d], [4, 3], 2, K, SEED)
+    grads = torch.zeros((K, plan.padded_elems), device="cuda")
+    draws = [[rng.laplace(size=d) * s for s in (1.0, 3.0, 0.2)], [rng.standard_t(3, size=d) * s for s in (0.5, 1.0, 2.0)]]
+    for m in range(2):
+        for k in range(K):
+            grads[k, plan.elem_offsets[m]: plan.elem_offsets[m] + d] = torch.from_numpy(draws[m][k].astype(np.float32)).cuda()
+    packed, norms, hist = plan.empty_packed(), plan.empty_norms(), plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels(hist, norms, K)
+    torch.cuda.synchronize()
+    N = norms.cpu().numpy().astype(np.float64)
+    for m, n in ((0, 16), (1, 8)):
+        lv = np.array(plan.lq_get_levels(m), np.float64)
+        assert lv[0] == 0 and lv[-1] == 1 and np.all(np.diff(lv) > 0)
+        v = grads[:, plan.elem_offsets[m]: plan.elem_offsets[m] + d].cpu().numpy().astype(np.float64)
+        u = np.minimum(np.abs(v) / N[:, m: m + 1], 1.0)
+        lam = N[:, m] ** 2 / np.sum(N[:, m] ** 2)
+
+        def variance(levels):
+            tau = np.clip(np.searchsorted(levels, u.ravel(), side="right") - 1, 0, len(levels) - 2).reshape(u.shape)
+            return float(np.sum(lam * np.mean((levels[tau + 1] - u) * (u - levels[tau]), axis=1)))
+        f_fit = variance(lv)
+        assert f_fit < variance(np.arange(n) / (n - 1.0))
+        assert f_fit < variance(np.concatenate([[0.0], 2.0 ** -np.arange(n - 2, -1, -1.0)]))
+        # (the fit sees the samples through 16 bins per octave: perturbations smaller than a bin can win by a hair)
+        for _ in range(60):
+            pert = lv.copy()
+            j = int(rng.integers(1, n - 1))
+            pert[j] += rng.choice([-1, 1]) * rng.uniform(0.1, 0.4) * min(pert[j] - pert[j - 1], pert[j + 1] - pert[j])
+            assert variance(pert) >= f_fit * (1 - 2e-3), (m, j)
+        for j in range(1, n - 1):
+            a, b, c = lv[j - 1], lv[j], lv[j + 1]
+            left = float(np.sum(lam * np.mean(np.where((u >= a) & (u < b), u - a, 0.0), axis=1)))
+            right = float(np.sum(lam * np.mean(np.where((u >= b) & (u < c), c - u, 0.0), axis=1)))
+            if min(((u >= a) & (u < b)).sum(), ((u >= b) & (u < c)).sum()) < 2000:
+                continue
+            assert abs(left - right) <= 0.03 * max(left, right), (m, j, left, right)
+
+
+def test_statistic_with_a_copy_of_the_previous_message(lqm, orc):
+    """prev_packed at another address than the buffer the last call wrote (a copy, a message that travelled), and
+    the same buffer after lq_message_modified: the plan may not skip words by what it remembers, and the statistic
+    and the update stay those of the oracle."""
+    sizes, K = [9000, 3000], 3
+    outs = []
+    for mode in ("same", "copy", "modified"):
+        plan = lqm.Plan(sizes, [4, 3], 2, K, SEED)
+        model = oracle_model(orc, plan)
+        X1 = _grads(plan, 5)[0].contiguous(); Y = torch.empty_like(X1); Xh = torch.empty_like(X1)
+        plan.qoda_init(X1, Y, Xh); model.qoda_init(to_unpadded(plan, X1))
+        pk = [plan.empty_packed(), plan.empty_packed()]; nm = [plan.empty_norms(), plan.empty_norms()]
+        for t in (1, 2, 3):
+            grads = _grads(plan, 300 + t)
+            grads[0, 1024:5000] = 0.0                                   # rows and blocks of zeros in one worker
+            if t == 2:
+                grads[1, :] = 0.0
+            c, p = t % 2, (t + 1) % 2
+            prev = pk[p]
+            if t > 1 and mode == "copy":
+                prev = pk[p].clone()
+            if t > 1 and mode == "modified":
+                pk[p].copy_(pk[p].clone())                              # rewritten in place (here: with the same words)
+                plan.lq_message_modified()
+            plan.lq_quantize_pack(grads, t, pk[c], nm[c], prev_packed=None if t == 1 else prev,
+                                  prev_norms=None if t == 1 else nm[p])
+            ref = model.quantize(to_unpadded(plan, grads), t)
+            assert compare_messages(orc, plan, pk[c], ref) == (0, 0)
+            sq, _ = plan.lq_get_statistics()
+            assert _close(sq.numpy(), ref["sq_diff"], 1e-12), (mode, t)
+            msg = pk[c]
+            if mode == "modified":
+                plan.lq_message_modified()
+            plan.qoda_step(msg, nm[c], X1, Y, Xh)
+            model.qoda_step()
+            assert _close(to_unpadded(plan, Y), model.Y, 1e-6) and _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
+        outs.append((Y.cpu().numpy().copy(), Xh.cpu().numpy().copy()))
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+    for a, b in zip(outs[0], outs[2]):
+        assert np.array_equal(a, b)
+
+
 def test_qoda_multi_step_small(lqm, orc):
     """20 iterations with random 'gradients' that depend on nothing: state parity every step."""
     sizes = [3000, 100, 2048]

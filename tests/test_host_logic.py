@@ -96,6 +96,19 @@ def test_two_gloo_ranks_take_the_max_time_and_sum_the_units(tmp_path):
         assert abs(r["value"] - 2 * 10.0 / 5e-3) < 1e-9           # all ranks' units / slowest rank's time
 
 
+def test_bench_gpus_n_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks by itself; with the stand-in step
+    (gloo, no GPU) rank 0 reports the world size, the slowest rank's time and the whole job's units."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--stub-step", "--steps", "3"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                        # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 2.0 and lines[0]["steps"] == 3
+    assert abs(lines[0]["value"] - 2 * 1.0 / 2e-3) < 1e-9
+
+
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2")
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2"],

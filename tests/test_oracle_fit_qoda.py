@@ -39,6 +39,25 @@ def test_uniform_density_gives_uniform_levels(orc):
         assert np.allclose(lv, np.arange(n) / (n - 1), atol=2e-4)
 
 
+def test_two_piece_density_has_levels_one_quarter_and_three_fifths(orc):
+    """A density that is constant on [0, 1/3] and 5/32 times as high on (1/3, 1].  With four levels {0, b1, b2, 1}
+    and b1 < 1/3 < b2 the two first-order conditions of the objective,
+        int_0^b1 u dF = int_b1^b2 (b2 - u) dF   and   int_b1^b2 (u - b1) dF = int_b2^1 (1 - u) dF,
+    read, with x = 1/3 - b1 and r = 5/32:
+        b1^2 / 2 = b2 x - ((1/3)^2 - b1^2) / 2 + r (b2 - 1/3)^2 / 2,
+        x^2 / 2 + r ((b2 - b1)^2 - x^2) / 2 = r (1 - b2)^2 / 2.
+    b1 = 1/4, b2 = 3/5 solve both exactly (worked out by hand: x = 1/12; 1/32 = 1/20 - 7/288 + (5/64)(16/225), and
+    (1/144)(27/32) = (5/32)(0.16 - 0.1225)), and a search from many starting points finds no other minimum."""
+    s, r = 1.0 / 3.0, 5.0 / 32.0
+    mass1 = s / (s + r * (1.0 - s))                              # share of the mass below 1/3
+    N = 1 << 22
+    q = (np.arange(N) + 0.5) / N                                 # the density's quantiles: an even sample of it
+    u = np.where(q < mass1, q / mass1 * s, s + (q - mass1) / (1.0 - mass1) * (1.0 - s))
+    lv = orc.fit_levels(_hist_of(orc, u)[None, :], [1.0], N, 4)
+    # (1/3 is not an edge of the histogram's bins, whose content is taken as evenly spread: 1e-3 of slack)
+    assert abs(lv[1] - 0.25) < 1e-3 and abs(lv[2] - 0.6) < 1e-3, lv
+
+
 @pytest.mark.parametrize("dist", ["halfnormal", "laplace", "student"])
 def test_fit_is_a_minimum_of_the_objective(orc, dist):
     rng = np.random.default_rng(42)

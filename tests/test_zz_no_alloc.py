@@ -47,6 +47,24 @@ def test_two_calls_in_a_row_match_the_plan_based_norm(q):
         assert abs(got - ref) <= 1e-6 * ref
 
 
+def test_calls_allocate_no_device_memory():
+    """What the entry point exists for: after a first call (which may load the library's module on the device),
+    further calls leave the device's free memory and torch's own allocation count unchanged."""
+    import paper_2505_14371_b200 as lqm
+    lqm.load_library()
+    v = torch.randn(3 * TILE + 5, device="cuda")
+    out = torch.zeros(1, device="cuda"); st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lqm.lq_vector_norm_static(v, 2, out, st)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0 = torch.cuda.memory_allocated()
+    for q in (2, 0, 1, 2):
+        lqm.lq_vector_norm_static(v, q, out, st)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_allocated() == held0
+
+
 def test_flags_limits_and_empty_input():
     import paper_2505_14371_b200 as lqm
     lib = lqm.load_library()
