@@ -83,6 +83,10 @@ def pick_workload(name: str):
         return W.transformer_xl_workload()
     if name == "wgan":
         return W.wgan_workload()
+    if name.startswith("wgan:"):                       # wgan:<bits>: the same shapes at another code width (Section 7.1 runs 5 bits)
+        w = W.wgan_workload()
+        w.bits = int(name.split(":")[1])
+        return w
     if name == "mlp":
         return W.mlp_workload()
     if name == "transformer_xl_small":
@@ -623,6 +627,72 @@ def run_sweep(args) -> None:
         del grads, pk, nm, X1, Y, Xh
 
 
+def run_entropy(args) -> None:
+    """Throughput of the entropy stage on one message of the chosen workload (appendix on the coding framework):
+    Huffman codes built from the message's own level counts, then lq_entropy_encode and lq_entropy_decode timed
+    with CUDA events (inputs resident, message larger than L2 or L2 flushed by a 256 MB write between
+    repetitions).  One JSON line: GB/s of the fixed-width message (K * W * 4 bytes), stream size, round trip."""
+    import torch
+    import paper_2505_14371_b200 as pkg
+    from paper_2505_14371_b200 import workloads as W
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    pkg.load_library()
+    w = pick_workload(args.workload)
+    K = w.num_workers
+    plan = pkg.Plan(w.layer_sizes, w.bits, w.q, K, W.PHILOX_SEED)
+    grads = W.make_gradients(w, plan.elem_offsets, plan.padded_elems, dev)
+    packed, norms, hist = plan.empty_packed(dev), plan.empty_norms(dev), plan.zero_hist(dev)
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels(hist, norms, K)
+    plan.lq_quantize_pack(grads, 2, packed, norms)
+    del grads, hist
+    counts = torch.zeros((K, plan.num_layers, 256), dtype=torch.int32, device=dev)
+    plan.lq_symbol_counts(packed, counts)
+    torch.cuda.synchronize()
+    tot = counts.sum(dim=0).cpu().numpy()
+    for m in range(plan.num_layers):
+        n = 1 << plan.bits[m]
+        plan.lq_code_set(m, pkg.lq_code_build([float(x) + 1e-9 for x in tot[m, :n]]))
+    Wd = plan.packed_words
+    stream = torch.zeros((K, Wd), dtype=torch.int32, device=dev)
+    offsets = torch.zeros((K, plan.lq_plan_blocks() + 1), dtype=torch.int32, device=dev)
+    back = torch.empty_like(packed)
+    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+    small = 4 * K * Wd < (256 << 20)
+    te, td = [], []
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for rep in range(args.steps + 3):
+        if small:
+            flush.fill_(float(rep))
+        ev[0].record()
+        plan.lq_entropy_encode(packed, stream, offsets)
+        ev[1].record()
+        if small:
+            flush.fill_(float(rep) + 0.5)
+        ev[2].record()
+        plan.lq_entropy_decode(stream, offsets, back)
+        ev[3].record()
+        torch.cuda.synchronize()
+        if rep >= 3:
+            te.append(ev[0].elapsed_time(ev[1])); td.append(ev[2].elapsed_time(ev[3]))
+    status = plan.lq_entropy_status()
+    words = offsets[:, -1].to(torch.int64).sum().item()
+    # a round trip returns the message with the sign bit of zero-index coordinates cleared: compare through a
+    # second encode of the decoded message, which must give the same stream
+    stream2 = torch.zeros_like(stream); offsets2 = torch.zeros_like(offsets)
+    plan.lq_entropy_encode(back, stream2, offsets2)
+    torch.cuda.synchronize()
+    same = bool(torch.equal(offsets, offsets2)) and bool(torch.equal(stream, stream2))
+    me, md = sorted(te)[len(te) // 2], sorted(td)[len(td) // 2]
+    msg_bytes = 4.0 * K * Wd
+    print(json.dumps({"entropy_stage": True, "workload": args.workload, "coords": w.num_coords, "num_workers": K, "bits": w.bits,
+                      "message_bytes": msg_bytes, "stream_bytes": 4.0 * words, "compression": msg_bytes / (4.0 * words),
+                      "encode_ms": me, "decode_ms": md, "encode_gbs": msg_bytes / me / 1e6, "decode_gbs": msg_bytes / md / 1e6,
+                      "status": status, "round_trip_same_stream": same,
+                      "l2": "flushed between repetitions" if small else "message exceeds L2"}), flush=True)
+
+
 def spawn_ranks(n: int, argv) -> int:
     """`python bench.py --gpus N` without a launcher: start N ranks of this script (one per GPU) under
     torch.distributed.run on this node and return their exit code."""
@@ -670,6 +740,7 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true", help="skip the extra dense-data measurement of the encoder (roofline.dense)")
     ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)   # launcher test: gloo ranks, no GPU work
+    ap.add_argument("--entropy", action="store_true", help="throughput of the entropy stage (encode / decode) on one message")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, widths, workers, norms")
     ap.add_argument("--sweep-quick", action="store_true")
     ap.add_argument("--sweep-bytes", type=float, default=40e9, help="most bytes of fp32 input per sweep point")
@@ -680,6 +751,9 @@ def main() -> None:
         return
     if args.sweep:
         run_sweep(args)
+        return
+    if args.entropy:
+        run_entropy(args)
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "ours" or args.stub_step):
         raise SystemExit(spawn_ranks(args.gpus, sys.argv[1:]))       # one process per GPU, started here

@@ -224,6 +224,66 @@ __device__ __forceinline__ double block_reduce(double v, double* scratch)
     return r;
 }
 
+// One value's term of a layer's L^q norm (Section 2.2), accumulated in fp64 (the maximum as an integer pattern).
+// mode 0: max |v|   1: sum |v|   2: sum v^2   3: sum |v|^q (integer q >= 3)
+template <int kMode>
+__device__ __forceinline__ void accumulate(double& acc, uint32_t& maxbits, float v, int q)
+{
+    if (kMode == 0) {
+        // |v| as an unsigned integer orders like the float; NaN and Inf have the largest patterns
+        const uint32_t b = __float_as_uint(v) & 0x7fffffffu;
+        maxbits = max(maxbits, b);
+    } else if (kMode == 1) {
+        acc += (double)fabsf(v);
+    } else if (kMode == 2) {
+        const double a = (double)v;
+        acc = fma(a, a, acc);            // the product of two floats is exact in fp64
+    } else {
+        const double a = fabs((double)v);
+        double p = a;
+        for (int r = 1; r < q; ++r) p = __dmul_rn(p, a);
+        acc += p;
+    }
+}
+
+// A layer's norm from the norm pass's partials, in a fixed order: thread i < 128 takes partials i, i + 128, ...,
+// then the CTA tree; the root, the rounding to fp32, the flags and the fp32 reciprocal.  Every thread of the CTA
+// calls it (128 threads or more); the result is valid in thread 0.  `scratch`: one double per warp.
+struct LayerNorm {
+    double total;        // the sum (or maximum) before the root
+    float norm, rnorm;   // fp32(||v||_q) and 1 / norm, both 0 when flagged
+    uint32_t status;
+    bool bad;            // a partial was NaN or Inf
+};
+__device__ __forceinline__ LayerNorm layer_norm_from_partials(const double* part, int n, int q, double* scratch)
+{
+    double acc = 0.0;
+    int bad = 0;
+    if (threadIdx.x < 128)
+        for (int i = threadIdx.x; i < n; i += 128) {
+            const double v = __ldcg(part + i);                   // (from L2: another CTA of this launch may have written it)
+            if (!(fabs(v) <= 1.7976931348623157e308)) bad = 1;
+            if (q == 0) acc = fmax(acc, v); else acc += v;
+        }
+    bad = __syncthreads_or(bad);
+    LayerNorm r;
+    r.total = q == 0 ? block_reduce<true>(acc, scratch) : block_reduce<false>(acc, scratch);
+    r.bad = bad != 0;
+    double n64;
+    if (q == 0 || q == 1) n64 = r.total;
+    else if (q == 2)      n64 = sqrt(r.total);
+    else                  n64 = pow(r.total, 1.0 / (double)q);
+    float nf = (float)n64;
+    r.status = 0;
+    if (bad || !(fabs(n64) <= 1.7976931348623157e308) || !(fabsf(nf) <= 3.402823466e38f))
+        r.status = LQ_STATUS_NONFINITE;
+    else if (nf < 1.17549435e-38f)
+        r.status = LQ_STATUS_ZERO_NORM;
+    r.norm = r.status ? 0.0f : nf;
+    r.rnorm = r.status ? 0.0f : __fdiv_rn(1.0f, nf);
+    return r;
+}
+
 #endif  // __CUDACC__
 
 }  // namespace lq

@@ -8,27 +8,6 @@
 
 namespace lq {
 
-// mode 0: max |v|   1: sum |v|   2: sum v^2   3: sum |v|^q (integer q >= 3)
-template <int kMode>
-__device__ __forceinline__ void accumulate(double& acc, uint32_t& maxbits, float v, int q)
-{
-    if (kMode == 0) {
-        // |v| as an unsigned integer orders like the float; NaN and Inf have the largest patterns
-        const uint32_t b = __float_as_uint(v) & 0x7fffffffu;
-        maxbits = max(maxbits, b);
-    } else if (kMode == 1) {
-        acc += (double)fabsf(v);
-    } else if (kMode == 2) {
-        const double a = (double)v;
-        acc = fma(a, a, acc);            // the product of two floats is exact in fp64
-    } else {
-        const double a = fabs((double)v);
-        double p = a;
-        for (int r = 1; r < q; ++r) p = __dmul_rn(p, a);
-        acc += p;
-    }
-}
-
 template <int kMode>
 __global__ void __launch_bounds__(kThreads) norm_partial_kernel(PlanDev p, const float* __restrict__ grads,
                                                                 bool write_mask)
@@ -104,35 +83,16 @@ __global__ void __launch_bounds__(128) norm_finalize_kernel(PlanDev p, float* __
     const int m = blockIdx.x, k = blockIdx.y + p.worker0;
     const LayerDesc L = p.layers[m];
     const double* part = p.norm_partial + ((int64_t)k * p.num_tiles + L.first_tile) * p.sub_tiles;
-    double acc = 0.0;
-    int bad = 0;
-    for (int i = threadIdx.x; i < L.ntiles * p.sub_tiles; i += blockDim.x) {
-        const double v = part[i];
-        if (!(fabs(v) <= 1.7976931348623157e308)) bad = 1;
-        if (p.q == 0) acc = fmax(acc, v); else acc += v;
-    }
-    bad = __syncthreads_or(bad);
-    const double total = p.q == 0 ? block_reduce<true>(acc, scratch) : block_reduce<false>(acc, scratch);
+    const LayerNorm r = layer_norm_from_partials(part, L.ntiles * p.sub_tiles, p.q, scratch);
     if (threadIdx.x == 0) {
         const int64_t o = (int64_t)k * p.num_layers + m;
         if (p.global_norm) {                     // the layers' totals are combined per worker by norm_global_kernel
-            p.layer_total[o] = bad ? __longlong_as_double(0x7ff8000000000000LL) : total;
+            p.layer_total[o] = r.bad ? __longlong_as_double(0x7ff8000000000000LL) : r.total;
             return;
         }
-        double n64;
-        if (p.q == 0 || p.q == 1) n64 = total;
-        else if (p.q == 2)        n64 = sqrt(total);
-        else                      n64 = pow(total, 1.0 / (double)p.q);
-        float n = (float)n64;
-        uint32_t st = 0;
-        if (bad || !(fabs(n64) <= 1.7976931348623157e308) || !(fabsf(n) <= 3.402823466e38f))
-            st = LQ_STATUS_NONFINITE;
-        else if (n < 1.17549435e-38f)
-            st = LQ_STATUS_ZERO_NORM;
-        if (st) n = 0.0f;
-        norms[o] = n;
-        p.rnorm[o] = st ? 0.0f : __fdiv_rn(1.0f, n);
-        p.status[o] = st;
+        norms[o] = r.norm;
+        p.rnorm[o] = r.rnorm;
+        p.status[o] = r.status;
     }
 }
 
