@@ -658,6 +658,7 @@ def run_entropy(args) -> None:
     stream = torch.zeros((K, Wd), dtype=torch.int32, device=dev)
     offsets = torch.zeros((K, plan.lq_plan_blocks() + 1), dtype=torch.int32, device=dev)
     back = torch.empty_like(packed)
+    runs = plan.empty_run_offsets(dev) if not args.no_run_offsets else None
     flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
     small = 4 * K * Wd < (256 << 20)
     te, td = [], []
@@ -666,12 +667,12 @@ def run_entropy(args) -> None:
         if small:
             flush.fill_(float(rep))
         ev[0].record()
-        plan.lq_entropy_encode(packed, stream, offsets)
+        plan.lq_entropy_encode(packed, stream, offsets, runs)
         ev[1].record()
         if small:
             flush.fill_(float(rep) + 0.5)
         ev[2].record()
-        plan.lq_entropy_decode(stream, offsets, back)
+        plan.lq_entropy_decode(stream, offsets, back, runs)
         ev[3].record()
         torch.cuda.synchronize()
         if rep >= 3:
@@ -689,7 +690,8 @@ def run_entropy(args) -> None:
     print(json.dumps({"entropy_stage": True, "workload": args.workload, "coords": w.num_coords, "num_workers": K, "bits": w.bits,
                       "message_bytes": msg_bytes, "stream_bytes": 4.0 * words, "compression": msg_bytes / (4.0 * words),
                       "encode_ms": me, "decode_ms": md, "encode_gbs": msg_bytes / me / 1e6, "decode_gbs": msg_bytes / md / 1e6,
-                      "status": status, "round_trip_same_stream": same,
+                      "status": status, "round_trip_same_stream": same, "run_offsets": runs is not None,
+                      "side_bytes": 0 if runs is None else 2.0 * runs.numel(),
                       "l2": "flushed between repetitions" if small else "message exceeds L2"}), flush=True)
 
 
@@ -741,6 +743,7 @@ def main() -> None:
     ap.add_argument("--no-dense", action="store_true", help="skip the extra dense-data measurement of the encoder (roofline.dense)")
     ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)   # launcher test: gloo ranks, no GPU work
     ap.add_argument("--entropy", action="store_true", help="throughput of the entropy stage (encode / decode) on one message")
+    ap.add_argument("--no-run-offsets", action="store_true", help="entropy stage without the run offsets (one thread decodes a block)")
     ap.add_argument("--sweep", action="store_true", help="bandwidth sweep over sizes, widths, workers, norms")
     ap.add_argument("--sweep-quick", action="store_true")
     ap.add_argument("--sweep-bytes", type=float, default=40e9, help="most bytes of fp32 input per sweep point")

@@ -268,20 +268,28 @@ int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* coun
  *                   [K][lq_plan_blocks() + 1] (first word of every block; the last entry is the worker's length in
  *                   words).  A worker whose stream does not fit keeps its offsets but loses the blocks that do not fit:
  *                   compare the last offset with capacity_words.  (W words always suffice for the flat code.)
+ *                   run_offsets: NULL, or dev [K][lq_plan_blocks()][LQ_CODE_RUNS] u16 that receives, for every block,
+ *                   the bit offsets inside the block's stream at which its LQ_CODE_RUNS = 8 runs of 128 coordinates
+ *                   (four lanes) start: side data of 16 bytes per block (1/8 bit per coordinate) that is not part of
+ *                   the stream and lets the decoder work on the eight runs of a block in parallel.
  *   lq_entropy_decode: the inverse, packed fully overwritten; it equals the encoded message except that the sign
  *                   bit of a coordinate with level index 0 comes back as 0 (the stream carries no sign there; the
- *                   decoded value is zero either way).  A stream with no valid word, or a block that runs past
- *                   its end, sets a flag that lq_entropy_status returns (and clears); nothing faults. */
+ *                   decoded value is zero either way).  With run_offsets (as written by lq_entropy_encode for this
+ *                   stream) one thread decodes each run, eight per block; with NULL one thread walks a whole block
+ *                   (an order of magnitude slower).  A stream with no valid word, a block that runs past its end,
+ *                   or a run that does not end where the next one starts, sets a flag that lq_entropy_status
+ *                   returns (and clears); nothing faults. */
 #define LQ_CODE_MAX_LEN 12
+#define LQ_CODE_RUNS    8
 int lq_code_build(const double* weights, int32_t n, uint8_t* lengths);
 int lq_code_universal(int32_t n, uint8_t* lengths);
 int lq_code_set(lq_plan* plan, int32_t layer, const uint8_t* lengths, int32_t n);
 int lq_code_get(lq_plan* plan, int32_t layer, uint8_t* lengths, int32_t n);
 int64_t lq_plan_blocks(const lq_plan* plan);        /* blocks of 1024 coordinates per worker, all layers */
 int lq_entropy_encode(lq_plan* plan, const uint32_t* packed, uint32_t* stream_words, int64_t capacity_words,
-                      uint32_t* block_offsets, void* stream);
+                      uint32_t* block_offsets, uint16_t* run_offsets, void* stream);
 int lq_entropy_decode(lq_plan* plan, const uint32_t* stream_words, int64_t capacity_words,
-                      const uint32_t* block_offsets, uint32_t* packed, void* stream);
+                      const uint32_t* block_offsets, const uint16_t* run_offsets, uint32_t* packed, void* stream);
 int lq_entropy_status(lq_plan* plan, uint32_t* host_flag);
 
 /* Ergodic average (the guarantees of Section 5 are stated for X-bar_{T+1/2} = sum_{t=1..T} X_{t+1/2} / T).

@@ -80,8 +80,8 @@ def load_library() -> C.CDLL:
     L.lq_code_set.argtypes = [vp, i32, u8p, i32]
     L.lq_code_get.argtypes = [vp, i32, u8p, i32]
     L.lq_plan_blocks.argtypes = [vp]; L.lq_plan_blocks.restype = i64
-    L.lq_entropy_encode.argtypes = [vp, vp, vp, i64, vp, vp]
-    L.lq_entropy_decode.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.lq_entropy_encode.argtypes = [vp, vp, vp, i64, vp, vp, vp]
+    L.lq_entropy_decode.argtypes = [vp, vp, i64, vp, vp, vp, vp]
     L.lq_entropy_status.argtypes = [vp, C.POINTER(u32)]
     L.lq_level_probabilities.argtypes = [vp, vp, vp, i32, i32, vp, vp]
     L.lq_symbol_counts.argtypes = [vp, vp, vp, vp]
@@ -286,13 +286,19 @@ class Plan:
     def lq_plan_blocks(self) -> int:
         return int(load_library().lq_plan_blocks(self._h))
 
-    def lq_entropy_encode(self, packed, stream_words, block_offsets) -> None:
+    def lq_entropy_encode(self, packed, stream_words, block_offsets, run_offsets=None) -> None:
         _check(load_library().lq_entropy_encode(self._h, _ptr(packed, torch.int32), _ptr(stream_words, torch.int32),
-                                                stream_words.shape[1], _ptr(block_offsets, torch.int32), _stream()))
+                                                stream_words.shape[1], _ptr(block_offsets, torch.int32),
+                                                _ptr(run_offsets, torch.int16), _stream()))
 
-    def lq_entropy_decode(self, stream_words, block_offsets, packed) -> None:
+    def lq_entropy_decode(self, stream_words, block_offsets, packed, run_offsets=None) -> None:
         _check(load_library().lq_entropy_decode(self._h, _ptr(stream_words, torch.int32), stream_words.shape[1],
-                                                _ptr(block_offsets, torch.int32), _ptr(packed, torch.int32), _stream()))
+                                                _ptr(block_offsets, torch.int32), _ptr(run_offsets, torch.int16),
+                                                _ptr(packed, torch.int32), _stream()))
+
+    def empty_run_offsets(self, device="cuda"):
+        """[K][blocks][8] int16 buffer for the run offsets of the entropy stage."""
+        return torch.zeros((self.num_workers, self.lq_plan_blocks(), 8), dtype=torch.int16, device=device)
 
     def lq_entropy_status(self) -> int:
         flag = C.c_uint32(0)

@@ -853,28 +853,30 @@ int lq_code_get(lq_plan* plan, int32_t layer, uint8_t* lengths, int32_t n)
 int64_t lq_plan_blocks(const lq_plan* plan) { return plan ? plan->dev.total_blocks : (int64_t)fail(LQ_EINVAL, "plan is NULL"); }
 
 int lq_entropy_encode(lq_plan* plan, const uint32_t* packed, uint32_t* stream_words, int64_t capacity_words,
-                      uint32_t* block_offsets, void* stream)
+                      uint32_t* block_offsets, uint16_t* run_offsets, void* stream)
 {
+    LQ_ALIGNED(run_offsets, 2);
     if (!plan || !packed || !stream_words || !block_offsets) return fail(LQ_EINVAL, "NULL argument");
     if (capacity_words < 0) return fail(LQ_EINVAL, "capacity_words < 0");
     LQ_ALIGNED(packed, 4); LQ_ALIGNED(stream_words, 4); LQ_ALIGNED(block_offsets, 4);
     const int rc = ensure_codes(plan);
     if (rc != LQ_OK) return rc;
     LQ_CUDA(launch_entropy_encode(plan->dev, packed, plan->d_code_enc, block_offsets, stream_words, capacity_words,
-                                  (cudaStream_t)stream));
+                                  run_offsets, (cudaStream_t)stream));
     return LQ_OK;
 }
 
 int lq_entropy_decode(lq_plan* plan, const uint32_t* stream_words, int64_t capacity_words,
-                      const uint32_t* block_offsets, uint32_t* packed, void* stream)
+                      const uint32_t* block_offsets, const uint16_t* run_offsets, uint32_t* packed, void* stream)
 {
+    LQ_ALIGNED(run_offsets, 2);
     if (!plan || !packed || !stream_words || !block_offsets) return fail(LQ_EINVAL, "NULL argument");
     if (capacity_words < 0) return fail(LQ_EINVAL, "capacity_words < 0");
     LQ_ALIGNED(packed, 4); LQ_ALIGNED(stream_words, 4); LQ_ALIGNED(block_offsets, 4);
     const int rc = ensure_codes(plan);
     if (rc != LQ_OK) return rc;
-    LQ_CUDA(launch_entropy_decode(plan->dev, stream_words, capacity_words, block_offsets, plan->d_code_dec, packed,
-                                  plan->d_code_bad, (cudaStream_t)stream));
+    LQ_CUDA(launch_entropy_decode(plan->dev, stream_words, capacity_words, block_offsets, run_offsets, plan->d_code_dec,
+                                  packed, plan->d_code_bad, (cudaStream_t)stream));
     return LQ_OK;
 }
 

@@ -118,7 +118,8 @@ template <int kModeWrite>
 __global__ void __launch_bounds__(kThreads) entropy_encode_kernel(PlanDev p, const uint32_t* __restrict__ packed,
                                                                   const uint32_t* __restrict__ enc_tables,
                                                                   uint32_t* __restrict__ offsets,
-                                                                  uint32_t* __restrict__ out, int64_t capacity)
+                                                                  uint32_t* __restrict__ out, int64_t capacity,
+                                                                  uint16_t* __restrict__ run_offsets)
 {
     __shared__ uint32_t enc[kMaxLevels];
     __shared__ uint32_t buf[kWarps][1056];
@@ -158,6 +159,10 @@ __global__ void __launch_bounds__(kThreads) entropy_encode_kernel(PlanDev p, con
         for (uint32_t i = lane; i < nwords; i += 32) buf[warp][i] = 0u;
         __syncwarp();
         uint32_t pos = incl - bits;
+        // where the runs of four lanes (128 coordinates) start inside the block's stream: lets a decoder work on
+        // eight runs of a block at once
+        if (run_offsets && (lane & 3) == 0)
+            run_offsets[((int64_t)k * p.total_blocks + L.block_off + blk) * LQ_CODE_RUNS + (lane >> 2)] = (uint16_t)pos;
         for (int pp = 0; pp < 32; ++pp) {
             if (!real_coord(blk, lane, pp, L.size)) continue;
             const uint32_t sym = symbol_at(w, C, pp), idx = sym >> 1;
@@ -245,23 +250,137 @@ __global__ void __launch_bounds__(128) entropy_decode_kernel(PlanDev p, const ui
     if (broken || wi - 2 > last) atomicOr(bad, 1u);           // no valid word, or the block ran past its end
 }
 
+// One thread per run of four lanes (128 coordinates) of a block, eight threads per block, one CTA per sub-tile
+// (32 blocks of one layer): every thread starts at its run's recorded bit offset and rebuilds its four lanes' words.
+// The decode table of the layer sits in shared memory.  A thread that meets no valid word, that would read past
+// the block's end, or that does not end where the next run starts reports a broken stream; nothing is read or
+// written out of bounds.
+template <int C>
+__device__ __forceinline__ void decode_run(const uint32_t* __restrict__ src, int64_t first, int64_t last, uint32_t start_bit,
+                                           uint32_t end_bit, bool check_end, const uint16_t* dec, int64_t blk, int run,
+                                           int64_t size, uint32_t* __restrict__ dst, bool& broken)
+{
+    int64_t wi = first + (start_bit >> 5);                    // next word to load
+    uint64_t window = 0;
+    int have = 0;                                             // valid bits in the low end of `window`
+    {
+        const uint32_t x = wi < last ? __ldg(src + wi) : 0u; ++wi;
+        window = (uint64_t)(x >> (start_bit & 31u));
+        have = 32 - (int)(start_bit & 31u);
+    }
+    uint32_t used = start_bit;
+    const bool full = (blk + 1) * kBlockCoords <= size;
+    // A run of 128 one-bit words "0" for level index 0 (what untouched rows turn into when 0 is the most frequent
+    // level): 128 zero bits, recognised without walking them.
+    if (full && check_end && end_bit - start_bit == 128u && dec[0] == (uint16_t)(1u << 8)) {
+        const int sh = (int)(start_bit & 31u);
+        const int64_t w0 = first + (start_bit >> 5);
+        uint32_t any = 0;
+        if (w0 + 4 + (sh ? 1 : 0) <= last) {
+            any = __ldg(src + w0) >> sh;
+#pragma unroll
+            for (int i = 1; i < 4; ++i) any |= __ldg(src + w0 + i);
+            if (sh) any |= __ldg(src + w0 + 4) << (32 - sh);
+            if (any == 0u) {
+                for (int l4 = 0; l4 < 4; ++l4)
+#pragma unroll
+                    for (int i = 0; i < C; ++i) dst[i * 32 + 4 * run + l4] = 0u;
+                return;
+            }
+        }
+    }
+    for (int l4 = 0; l4 < 4; ++l4) {
+        const int lane = 4 * run + l4;
+        uint32_t cw[C + 1];
+#pragma unroll
+        for (int i = 0; i <= C; ++i) cw[i] = 0u;
+#pragma unroll
+        for (int pp = 0; pp < 32; ++pp) {
+            if (!full && !(blk * kBlockCoords + 128 * (pp >> 2) + 4 * lane + (pp & 3) < size)) continue;
+            if (have <= 32) { const uint32_t x = wi < last ? __ldg(src + wi) : 0u; ++wi; window |= (uint64_t)x << have; have += 32; }
+            const uint32_t e = dec[window & ((1u << kCodeMaxLen) - 1u)];
+            if (e == 0xffffu) { broken = true; continue; }
+            const uint32_t idx = e & 0xffu, l = e >> 8;
+            window >>= l; have -= (int)l; used += l;
+            uint32_t sym = idx << 1;
+            if (idx != 0u) { sym |= (uint32_t)(window & 1u); window >>= 1; have -= 1; used += 1u; }
+            const int off = pp * C, i = off >> 5, s = off & 31;
+            cw[i] |= sym << s;
+            if (s + C > 32) cw[i + 1] |= sym >> (32 - s);
+        }
+#pragma unroll
+        for (int i = 0; i < C; ++i) dst[i * 32 + lane] = cw[i];
+    }
+    if (check_end ? used != end_bit : ((int64_t)((used + 31u) >> 5) > last - first)) broken = true;
+}
+
+__global__ void __launch_bounds__(kThreads) entropy_decode_runs_kernel(PlanDev p, const uint32_t* __restrict__ in, int64_t capacity,
+                                                                       const uint32_t* __restrict__ offsets,
+                                                                       const uint16_t* __restrict__ run_offsets,
+                                                                       const uint16_t* __restrict__ dec_tables,
+                                                                       uint32_t* __restrict__ packed, uint32_t* __restrict__ bad)
+{
+    __shared__ uint16_t dec[1 << kCodeMaxLen];
+    const Tile tile = p.tiles[blockIdx.x >> p.sub_shift];
+    const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
+    if (sub0 >= tile.nblocks) return;
+    const int layer = tile.layer, k = blockIdx.y;
+    const LayerDesc L = p.layers[layer];
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(dec_tables + ((int64_t)layer << kCodeMaxLen));
+        uint4* dst = reinterpret_cast<uint4*>(dec);
+        for (int i = threadIdx.x; i < (1 << kCodeMaxLen) / 8; i += blockDim.x) dst[i] = __ldg(src + i);
+    }
+    __syncthreads();
+    const int b = sub0 + (threadIdx.x >> 3), run = threadIdx.x & 7;
+    if (b >= tile.nblocks) return;
+    const int64_t blk = tile.block0 + b, g = L.block_off + blk;
+    const uint32_t* off_k = offsets + (int64_t)k * (p.total_blocks + 1);
+    const int64_t first = off_k[g], last = min((int64_t)off_k[g + 1], capacity);
+    const uint16_t* ro = run_offsets + ((int64_t)k * p.total_blocks + g) * LQ_CODE_RUNS;
+    const uint32_t start_bit = ro[run];
+    const uint32_t end_bit = run + 1 < LQ_CODE_RUNS ? (uint32_t)ro[run + 1] : 0u;
+    const int C = L.bits + 1;
+    uint32_t* dst = packed + (int64_t)k * p.packed_words + L.word_off + blk * (int64_t)C * 32;
+    const uint32_t* src = in + (int64_t)k * capacity;
+    bool broken = first + (start_bit >> 5) > last;            // an offset that points past the block's end
+    if (broken) {                                             // the run's words are still written (zeros), nothing is read
+        for (int l4 = 0; l4 < 4; ++l4)
+            for (int i = 0; i < C; ++i) dst[i * 32 + 4 * run + l4] = 0u;
+    } else {
+        switch (C) {
+#define LQ_CASE(CC) case CC: decode_run<CC>(src, first, last, start_bit, end_bit, run + 1 < LQ_CODE_RUNS, dec, blk, run, L.size, dst, broken); break;
+            LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8) LQ_CASE(9)
+#undef LQ_CASE
+            default: break;
+        }
+    }
+    if (broken) atomicOr(bad, 1u);
+}
+
 }  // namespace
 
 cudaError_t launch_entropy_encode(const PlanDev& p, const uint32_t* packed, const uint32_t* enc_tables,
-                                  uint32_t* offsets, uint32_t* out, int64_t capacity, cudaStream_t s)
+                                  uint32_t* offsets, uint32_t* out, int64_t capacity, uint16_t* run_offsets, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
     const dim3 grid((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.num_workers);
-    entropy_encode_kernel<0><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity);
+    entropy_encode_kernel<0><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, nullptr);
     entropy_scan_kernel<<<(unsigned)p.num_workers, 1024, 0, s>>>(p, offsets);
-    entropy_encode_kernel<1><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity);
+    entropy_encode_kernel<1><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, run_offsets);
     return cudaGetLastError();
 }
 
 cudaError_t launch_entropy_decode(const PlanDev& p, const uint32_t* in, int64_t capacity, const uint32_t* offsets,
-                                  const uint16_t* dec_tables, uint32_t* packed, uint32_t* bad, cudaStream_t s)
+                                  const uint16_t* run_offsets, const uint16_t* dec_tables, uint32_t* packed, uint32_t* bad,
+                                  cudaStream_t s)
 {
     if (p.total_blocks == 0) return cudaSuccess;
+    if (run_offsets) {
+        const dim3 grid_r((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.num_workers);
+        entropy_decode_runs_kernel<<<grid_r, kThreads, 0, s>>>(p, in, capacity, offsets, run_offsets, dec_tables, packed, bad);
+        return cudaGetLastError();
+    }
     const dim3 grid((unsigned)((p.total_blocks + 127) / 128), (unsigned)p.num_workers);
     entropy_decode_kernel<<<grid, 128, 0, s>>>(p, in, capacity, offsets, dec_tables, packed, bad);
     return cudaGetLastError();

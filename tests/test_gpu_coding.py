@@ -88,6 +88,43 @@ def test_stream_matches_the_oracle_and_round_trips(lqm, orc, bits):
     torch.cuda.synchronize()
     assert plan.lq_entropy_status() == 0
     assert np.array_equal(back.cpu().numpy().view(np.uint32), _canonical(orc, plan, packed))
+    # the run offsets (side data for the parallel decoder): for run r of a block, the bits of the coordinates that
+    # precede it in the block's stream order s = 32 lane + p, from the definition; the stream itself is unchanged
+    runs = plan.empty_run_offsets()
+    stream2 = torch.full_like(stream, -1); offs2 = torch.zeros_like(offs)
+    plan.lq_entropy_encode(packed, stream2, offs2, runs)
+    torch.cuda.synchronize()
+    assert torch.equal(offs, offs2)
+    R = runs.cpu().numpy().view(np.uint16)
+    for k in range(plan.num_workers):
+        assert np.array_equal(stream2[k, : O[k, -1]].cpu().numpy(), stream[k, : O[k, -1]].cpu().numpy())
+        g = 0
+        for m, d in enumerate(sizes):
+            l = np.array(lengths[m], np.int64)
+            for blk in range((d + 1023) // 1024):
+                ss = np.arange(1024); lane, pp = ss // 32, ss % 32
+                coord = blk * 1024 + 128 * (pp // 4) + 4 * lane + pp % 4          # coordinate of stream position s
+                real = coord < d
+                ix = np.zeros(1024, np.int64); ix[real] = ref["idx"][k, off[m] + coord[real]]
+                nbits = np.where(real, l[ix] + (ix != 0), 0)
+                want = np.concatenate([[0], np.cumsum(nbits)])[0:1024:128]
+                assert np.array_equal(R[k, g].astype(np.int64), want), (k, m, blk)
+                g += 1
+    back2 = torch.full_like(packed, -1)
+    plan.lq_entropy_decode(stream, offs, back2, runs)
+    torch.cuda.synchronize()
+    assert plan.lq_entropy_status() == 0
+    assert torch.equal(back2, back)
+    # offsets that do not belong to the stream are reported, never followed out of bounds
+    bad_runs = runs.clone(); bad_runs[:, :, 3] += 1
+    plan.lq_entropy_decode(stream, offs, back2, bad_runs)
+    torch.cuda.synchronize()
+    if plan.lq_plan_blocks() > 0:
+        assert plan.lq_entropy_status() != 0
+    wild = torch.full_like(runs, 32767)
+    plan.lq_entropy_decode(stream, offs, back2, wild)
+    torch.cuda.synchronize()
+    assert plan.lq_entropy_status() != 0 and plan.lq_entropy_status() == 0
     # what the decoder rebuilds decodes to the same values
     g1 = torch.empty(plan.padded_elems, device="cuda"); g2 = torch.empty_like(g1)
     plan.lq_decode_aggregate(packed, norms, g1); plan.lq_decode_aggregate(back, norms, g2)
