@@ -358,3 +358,24 @@ def test_shared_fit_reduces_to_the_single_layer_fit_and_minimises_the_summed_var
         j = int(rng.integers(1, 15))
         p[j] += rng.uniform(-0.3, 0.3) * min(p[j] - p[j - 1], p[j + 1] - p[j])
         assert best <= total_variance(p) * 1.002
+
+
+def test_fp32_difference_costs_less_than_one_ulp_in_the_statistic(orc):
+    """The statistic of Eq. (general_stepsize) takes the difference of two decoded fp32 values in fp32 (one rounding)
+    before squaring in fp64.  Against the exact difference (both values converted to fp64 first) every term is off by at
+    most a relative 2^-23, and so is the sum; on two successive messages of normal data the sums differ by far less."""
+    rng = np.random.default_rng(11)
+    d = 200000
+    lv = orc.uniform_levels(4)
+    decoded = []
+    for step, scale in ((1, 1.0), (2, 0.8)):
+        v = (rng.standard_normal(d) * scale).astype(np.float32)
+        norm, _ = orc.layer_norm(v, 2)
+        idx, sg, _ = orc.quantize_layer(v, norm, lv, 7, step, 0, 0)
+        decoded.append(orc.decode_layer(idx, sg, norm, lv))
+    got = orc.sq_diff(decoded[1], decoded[0])
+    exact = float(np.sum((decoded[1].astype(np.float64) - decoded[0].astype(np.float64)) ** 2))
+    rel = abs(got - exact) / exact
+    assert rel <= 2.0 ** -23
+    assert rel <= 1e-7, rel
+    print("relative cost of the fp32 difference in the statistic:", rel)
