@@ -229,7 +229,10 @@ void orc_histogram_layer(const float* v, int64_t d, float norm, uint32_t* hist)
  * The paper names no solver; this one is this implementation's own ("parity unpinned"):
  *   F~ is taken piecewise linear from the merged histogram (uniform density in a bin);
  *   the mass at u = 1 (last bin) never contributes variance and is left out;
- *   start: quantiles j/(n-1) of the mass above bin 0;
+ *   two starts, each followed by the sweeps below: (A) quantiles j/(n-1) of the mass above bin 0,
+ *     (B) the uniform grid j/(n-1).  Coordinate descent stops at a local minimum and the objective
+ *     has several when the density is not log-concave; the result is the start whose end point has
+ *     the smaller objective, B only if it is smaller by more than one part in 10^9;
  *   sweeps: exact coordinate minimisation of one interior level given its neighbours
  *     a < c, i.e. F~(l) = F~(c) - int_a^c (u-a)/(c-a) dF~(u)  (the first-order condition
  *     int_a^l (u-a) dF~ = int_l^c (c-u) dF~), odd levels first, then even levels;
@@ -244,6 +247,7 @@ typedef struct {
     double mass[ORC_NUM_BINS];        /* weighted mass of bins 0..384 (bin 385 unused) */
     double F[ORC_NUM_BINS + 1];       /* cumulative mass at the edges */
     double M1[ORC_NUM_BINS + 1];      /* cumulative first moment at the edges */
+    double M2[ORC_NUM_BINS + 1];      /* cumulative second moment at the edges */
 } orc_density;
 
 static int find_bin(const orc_density* D, double x)
@@ -277,6 +281,30 @@ static double cdf_inverse(const orc_density* D, double y)
     double t = (y - D->F[lo]) / D->mass[lo];
     if (t < 0.0) t = 0.0;
     return D->e[lo] + t * (D->e[lo + 1] - D->e[lo]);
+}
+
+/* int_0^x u^2 dF~(u): inside a bin of density m/(e1-e0), int_{e0}^{x} u^2 = part * (e0^2 + e0 x + x^2) / 3 */
+static double second_moment_at(const orc_density* D, double x)
+{
+    int i = find_bin(D, x);
+    double theta = (x - D->e[i]) / (D->e[i + 1] - D->e[i]);
+    if (theta > 1.0) theta = 1.0;
+    double part = D->mass[i] * theta;
+    return D->M2[i] + part * ((D->e[i] * D->e[i] + D->e[i] * x + x * x) / 3.0);
+}
+
+/* sum_j int_{l_j}^{l_{j+1}} (l_{j+1} - u)(u - l_j) dF~(u) from the cumulative moments:
+ * each interval gives -(M2(c) - M2(a)) + (a + c)(M1(c) - M1(a)) - a c (F(c) - F(a)). */
+static double density_objective(const orc_density* D, const double* l, int n)
+{
+    double total = 0.0;
+    for (int j = 0; j + 1 < n; ++j) {
+        double a = l[j], c = l[j + 1], m1a, m1c;
+        double Fa = cdf_at(D, a, &m1a), Fc = cdf_at(D, c, &m1c);
+        double m2a = second_moment_at(D, a), m2c = second_moment_at(D, c);
+        total += ((a + c) * (m1c - m1a) - (m2c - m2a)) - (a * c) * (Fc - Fa);
+    }
+    return total;
 }
 
 static orc_density D;                 /* single-threaded oracle: static storage is fine */
@@ -324,22 +352,9 @@ int orc_fit_levels_shared(const uint32_t* hist, int64_t stride, const float* nor
     return solve_levels(n, level_out);
 }
 
-/* The solver proper, on the density left in D. */
-static int solve_levels(int n, float* level_out)
+/* Odd/even sweeps of exact coordinate minimisation from the levels in l. */
+static void descend(double* l, int n)
 {
-    D.F[0] = 0.0; D.M1[0] = 0.0;
-    for (int i = 0; i < 385; ++i) {
-        D.F[i + 1] = D.F[i] + D.mass[i];
-        D.M1[i + 1] = D.M1[i] + D.mass[i] * ((D.e[i] + D.e[i + 1]) * 0.5);
-    }
-    double total = D.F[385], above = total - D.mass[0];
-    if (!(above > 0.0)) return 0;
-
-    double l[256];
-    l[0] = 0.0; l[n - 1] = 1.0;
-    for (int j = 1; j <= n - 2; ++j)
-        l[j] = cdf_inverse(&D, D.mass[0] + above * ((double)j / (double)(n - 1)));
-
     for (int sweep = 0; sweep < 100; ++sweep) {
         double moved = 0.0;
         for (int parity = 1; parity >= 0; --parity) {
@@ -364,6 +379,32 @@ static int solve_levels(int n, float* level_out)
         }
         if (moved <= 1e-13) break;
     }
+}
+
+/* The solver proper, on the density left in D. */
+static int solve_levels(int n, float* level_out)
+{
+    D.F[0] = 0.0; D.M1[0] = 0.0; D.M2[0] = 0.0;
+    for (int i = 0; i < 385; ++i) {
+        D.F[i + 1] = D.F[i] + D.mass[i];
+        D.M1[i + 1] = D.M1[i] + D.mass[i] * ((D.e[i] + D.e[i + 1]) * 0.5);
+        D.M2[i + 1] = D.M2[i] + D.mass[i] * ((D.e[i] * D.e[i] + D.e[i] * D.e[i + 1] + D.e[i + 1] * D.e[i + 1]) / 3.0);
+    }
+    double total = D.F[385], above = total - D.mass[0];
+    if (!(above > 0.0)) return 0;
+
+    double l[256], lb[256];
+    l[0] = 0.0; l[n - 1] = 1.0;
+    lb[0] = 0.0; lb[n - 1] = 1.0;
+    for (int j = 1; j <= n - 2; ++j) {
+        l[j] = cdf_inverse(&D, D.mass[0] + above * ((double)j / (double)(n - 1)));
+        lb[j] = (double)j / (double)(n - 1);
+    }
+    descend(l, n);
+    descend(lb, n);
+    double obj_a = density_objective(&D, l, n), obj_b = density_objective(&D, lb, n);
+    if (obj_b < obj_a * (1.0 - 1e-9))
+        for (int j = 1; j <= n - 2; ++j) l[j] = lb[j];
 
     level_out[0] = 0.0f; level_out[n - 1] = 1.0f;
     for (int j = 1; j <= n - 2; ++j) {
