@@ -181,7 +181,10 @@ int lq_quantize_pack(lq_plan* plan, const float* grads, uint32_t step, uint32_t*
  * CDF weights lambda_z = N_z^2 / sum N_z^2): for every layer with at least 3 levels, merge
  * the num_samples histograms of that layer with those weights and minimise
  * sum_j int_{l_j}^{l_{j+1}} (l_{j+1}-u)(u-l_j) dF~(u) by exact coordinate minimisation
- * (the solver is this library's: the paper states the objective only).
+ * (the solver is this library's: the paper states the objective only).  The descent runs from two
+ * starts, the quantiles of the merged mass and the uniform grid, and the end point with the smaller
+ * objective is kept; the result is a stationary point, for a density that is not log-concave not
+ * necessarily the global minimum.
  *   hist dev [num_samples][L][LQ_HIST_STRIDE];  norms dev [num_samples][L].
  * The new levels are staged: they take effect at the next lq_quantize_pack.  Layers with no
  * usable mass keep their levels. */

@@ -6,6 +6,11 @@
 // l solves  F~(l) = F~(c) - int_a^c (u - a)/(c - a) dF~(u).  F~ is piecewise linear (uniform density
 // inside a histogram bin), so F~, its first moment and its inverse are closed forms.
 //
+// Coordinate descent stops at a local minimum, and the objective has several when the density is not log-concave
+// (a step density already has two), so the descent runs from two starts, the quantiles of the mass above bin 0 and the
+// uniform grid, and the end point with the smaller objective is kept (the uniform start's only if it is smaller by
+// more than one part in 10^9, so that rounding does not decide between two copies of the same minimum).
+//
 // One CTA per layer; odd and even interior levels are updated in two parallel half-sweeps (levels of
 // one parity only depend on the other parity).  All arithmetic is fp64 and this file is compiled
 // without FMA contraction so that the sequence of roundings is the plain one.
@@ -22,7 +27,11 @@ struct FitSmem {
     double mass[kBins];
     double F[kBins + 1];
     double M1[kBins + 1];
+    double M2[kBins + 1];
     double l[kMaxLevels];
+    double lb[kMaxLevels];
+    double term[kMaxLevels];
+    double obj[2];
     double lambda[LQ_MAX_WORKERS];
     double red[kFitThreads / 32];
     double moved;
@@ -56,6 +65,16 @@ __device__ double cdf(const FitSmem& s, double x, double* m1)
     return s.F[i] + part;
 }
 
+// int_0^x u^2 dF~(u); inside a bin int_{e0}^{x} u^2 = (mass in [e0, x]) * (e0^2 + e0 x + x^2) / 3
+__device__ double second_moment(const FitSmem& s, double x)
+{
+    const int i = bin_of(s, x);
+    double theta = (x - s.e[i]) / (s.e[i + 1] - s.e[i]);
+    if (theta > 1.0) theta = 1.0;
+    const double part = s.mass[i] * theta;
+    return s.M2[i] + part * ((s.e[i] * s.e[i] + s.e[i] * x + x * x) / 3.0);
+}
+
 __device__ double cdf_inv(const FitSmem& s, double y)
 {
     int lo = 0, hi = kBins;
@@ -67,6 +86,66 @@ __device__ double cdf_inv(const FitSmem& s, double y)
     double t = (y - s.F[lo]) / s.mass[lo];
     if (t < 0.0) t = 0.0;
     return s.e[lo] + t * (s.e[lo + 1] - s.e[lo]);
+}
+
+// Odd/even sweeps of exact coordinate minimisation on the levels l (shared memory), by the whole CTA.
+__device__ void descend(FitSmem& s, double* l, int n, int tid)
+{
+    for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
+        double moved = 0.0;
+        for (int parity = 1; parity >= 0; --parity) {
+            for (int j = tid; j <= n - 2; j += kFitThreads) {
+                if (j < 1 || (j & 1) != parity) continue;
+                const double a = l[j - 1], c = l[j + 1];
+                if (!(c > a)) continue;
+                double m1a, m1c, b;
+                const double Fa = cdf(s, a, &m1a), Fc = cdf(s, c, &m1c);
+                const double mass_ac = Fc - Fa;
+                if (!(mass_ac > 0.0)) b = (a + c) * 0.5;
+                else {
+                    const double target = Fc - ((m1c - m1a) - a * mass_ac) / (c - a);
+                    b = cdf_inv(s, target);
+                    if (b < a) b = a;
+                    if (b > c) b = c;
+                }
+                const double rel = fabs(b - l[j]) / (fabs(b) > 1e-300 ? fabs(b) : 1e-300);
+                if (rel > moved) moved = rel;
+                l[j] = b;
+            }
+            __syncthreads();
+        }
+        moved = warp_max(moved);
+        if ((tid & 31) == 0) s.red[tid >> 5] = moved;
+        __syncthreads();
+        if (tid == 0) {
+            double mx = s.red[0];
+            for (int w = 1; w < kFitThreads / 32; ++w) mx = fmax(mx, s.red[w]);
+            s.moved = mx;
+        }
+        __syncthreads();
+        if (s.moved <= 1e-13) break;
+    }
+    __syncthreads();
+}
+
+// The objective at the levels l: interval j gives -(M2(c) - M2(a)) + (a + c)(M1(c) - M1(a)) - a c (F(c) - F(a));
+// the intervals are added in order by one thread so that the sum does not depend on the CTA's shape.
+__device__ void objective(FitSmem& s, const double* l, int n, int tid, double* out)
+{
+    for (int j = tid; j + 1 < n; j += kFitThreads) {
+        const double a = l[j], c = l[j + 1];
+        double m1a, m1c;
+        const double Fa = cdf(s, a, &m1a), Fc = cdf(s, c, &m1c);
+        const double m2a = second_moment(s, a), m2c = second_moment(s, c);
+        s.term[j] = ((a + c) * (m1c - m1a) - (m2c - m2a)) - (a * c) * (Fc - Fa);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double total = 0.0;
+        for (int j = 0; j + 1 < n; ++j) total += s.term[j];
+        *out = total;
+    }
+    __syncthreads();
 }
 
 // Per-layer mode (member_off == nullptr): CTA m fits layer m.  Shared mode: CTA t fits one sequence for type t,
@@ -145,10 +224,11 @@ __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, cons
     __syncthreads();
     }
     if (tid == 0) {
-        s.F[0] = 0.0; s.M1[0] = 0.0;
+        s.F[0] = 0.0; s.M1[0] = 0.0; s.M2[0] = 0.0;
         for (int i = 0; i < kBins; ++i) {
             s.F[i + 1] = s.F[i] + s.mass[i];
             s.M1[i + 1] = s.M1[i] + s.mass[i] * ((s.e[i] + s.e[i + 1]) * 0.5);
+            s.M2[i + 1] = s.M2[i] + s.mass[i] * ((s.e[i] * s.e[i] + s.e[i] * s.e[i + 1] + s.e[i + 1] * s.e[i + 1]) / 3.0);
         }
         s.ok = (s.F[kBins] - s.mass[0]) > 0.0;
     }
@@ -157,46 +237,23 @@ __global__ void __launch_bounds__(kFitThreads) fit_levels_kernel(PlanDev p, cons
 
     const double above = s.F[kBins] - s.mass[0];
     for (int j = tid; j < n; j += kFitThreads) {
-        if (j == 0) s.l[j] = 0.0;
-        else if (j == n - 1) s.l[j] = 1.0;
-        else s.l[j] = cdf_inv(s, s.mass[0] + above * ((double)j / (double)(n - 1)));
+        const double frac = (double)j / (double)(n - 1);
+        if (j == 0) s.l[j] = s.lb[j] = 0.0;
+        else if (j == n - 1) s.l[j] = s.lb[j] = 1.0;
+        else {
+            s.l[j] = cdf_inv(s, s.mass[0] + above * frac);
+            s.lb[j] = frac;
+        }
     }
     __syncthreads();
 
-    for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
-        double moved = 0.0;
-        for (int parity = 1; parity >= 0; --parity) {
-            for (int j = tid; j <= n - 2; j += kFitThreads) {
-                if (j < 1 || (j & 1) != parity) continue;
-                const double a = s.l[j - 1], c = s.l[j + 1];
-                if (!(c > a)) continue;
-                double m1a, m1c, b;
-                const double Fa = cdf(s, a, &m1a), Fc = cdf(s, c, &m1c);
-                const double mass_ac = Fc - Fa;
-                if (!(mass_ac > 0.0)) b = (a + c) * 0.5;
-                else {
-                    const double target = Fc - ((m1c - m1a) - a * mass_ac) / (c - a);
-                    b = cdf_inv(s, target);
-                    if (b < a) b = a;
-                    if (b > c) b = c;
-                }
-                const double rel = fabs(b - s.l[j]) / (fabs(b) > 1e-300 ? fabs(b) : 1e-300);
-                if (rel > moved) moved = rel;
-                s.l[j] = b;
-            }
-            __syncthreads();
-        }
-        moved = warp_max(moved);
-        if ((tid & 31) == 0) s.red[tid >> 5] = moved;
-        __syncthreads();
-        if (tid == 0) {
-            double mx = s.red[0];
-            for (int w = 1; w < kFitThreads / 32; ++w) mx = fmax(mx, s.red[w]);
-            s.moved = mx;
-        }
-        __syncthreads();
-        if (s.moved <= 1e-13) break;
-    }
+    descend(s, s.l, n, tid);
+    descend(s, s.lb, n, tid);
+    objective(s, s.l, n, tid, &s.obj[0]);
+    objective(s, s.lb, n, tid, &s.obj[1]);
+    if (s.obj[1] < s.obj[0] * (1.0 - 1e-9))
+        for (int j = 1 + tid; j <= n - 2; j += kFitThreads) s.l[j] = s.lb[j];
+    __syncthreads();
 
     // round to fp32; force strict monotonicity (one ulp and 2^-40 above the level before, one ulp
     // below the level after; serial: order matters)

@@ -288,6 +288,32 @@ def test_fitted_levels_minimise_the_variance_on_the_samples(lqm):
             assert abs(left - right) <= 0.04 * max(left, right), (m, j, left, right)
 
 
+def test_fit_ends_in_the_lower_of_two_minima(lqm, orc):
+    """A density constant on [0, 3/11] and 4/125 as high above has, with four levels, two local minima of the fit's
+    objective; (1/5, 1/2) satisfies both first-order conditions and is the lower one (the CPU suite finds it by brute
+    force), the quantile start alone ends near (0.136, 0.272).  Max norm, so that u is the value itself."""
+    s, r = 3.0 / 11.0, 4.0 / 125.0
+    mass1 = s / (s + r * (1.0 - s))
+    N = 1 << 22
+    q = (np.arange(N) + 0.5) / N
+    u = np.where(q < mass1, q / mass1 * s, s + (q - mass1) / (1.0 - mass1) * (1.0 - s)).astype(np.float32)
+    v = np.concatenate([u, np.float32([1.0])])
+    v[1::2] *= -1
+    plan = lqm.Plan([v.size], [2], 0, 1, SEED)
+    grads = torch.zeros((1, plan.padded_elems), device="cuda")
+    grads[0, : v.size] = torch.from_numpy(v).cuda()
+    packed, norms, hist = plan.empty_packed(), plan.empty_norms(), plan.zero_hist()
+    plan.lq_quantize_pack(grads, 1, packed, norms, hist=hist)
+    plan.lq_fit_levels(hist, norms, 1)
+    got = np.array(plan.lq_get_levels(0))
+    assert norms.cpu().numpy().ravel()[0] == 1.0
+    # (the step at 3/11 is smeared over the histogram bin [17/64, 18/64]: a few 1e-3 of slack)
+    assert abs(got[1] - 0.2) < 2e-3 and abs(got[2] - 0.5) < 4e-3, got
+    h = hist.cpu().numpy().view(np.uint32)
+    want = orc.fit_levels(h[:, 0, :], norms.cpu().numpy()[:, 0], v.size, 4)
+    assert np.allclose(got, want, rtol=1e-6, atol=0)
+
+
 def test_statistic_with_a_copy_of_the_previous_message(lqm, orc):
     """prev_packed at another address than the buffer the last call wrote (a copy, a message that travelled), and
     the same buffer after lq_message_modified: the plan may not skip words by what it remembers, and the statistic
