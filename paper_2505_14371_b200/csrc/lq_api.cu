@@ -70,7 +70,7 @@ struct lq_plan {
     uint64_t seed = 0;
     LayerDesc* d_layers = nullptr;
     Tile* d_tiles = nullptr;
-    int32_t* d_tile_order = nullptr;
+    TileJob* d_jobs = nullptr;
     float* d_levels_stage = nullptr;
     float* d_levels_enc[2] = {nullptr, nullptr};
     SearchTables search{};         // derived from d_levels_enc[cur]
@@ -105,9 +105,9 @@ namespace {
 void free_plan(lq_plan* p)
 {
     if (!p) return;
-    cudaFree(p->d_layers); cudaFree(p->d_tiles); cudaFree(p->d_tile_order);
+    cudaFree(p->d_layers); cudaFree(p->d_tiles); cudaFree(p->d_jobs);
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
-    cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast); cudaFree(p->search.first);
+    cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
     cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     cudaFree(p->dev.block_live);
@@ -251,7 +251,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     const size_t lev = (size_t)(num_layers ? num_layers : 1) * kLevelStride;
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_layers, p->layers.size());
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_tiles, p->tiles.size());
-    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_tile_order, p->tiles.size());
+    if (e == cudaSuccess) e = dev_alloc_zero(&p->d_jobs, p->tiles.size());
     if (e == cudaSuccess && !p->tiles.empty()) {
         // the encoder's launch order: tiles sorted by their relative position inside their layer, so that every
         // layer is under way from the first wave of CTAs to the last
@@ -268,7 +268,16 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
             const int64_t kb = (2 * (int64_t)(b - Lb.first_tile) + 1) * La.ntiles;
             return ka != kb ? ka < kb : a < b;
         });
-        e = cudaMemcpy(p->d_tile_order, order.data(), order.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+        std::vector<TileJob> jobs;
+        try { jobs.resize(order.size()); } catch (const std::bad_alloc&) { free_plan(p); return fail(LQ_ENOMEM, "host allocation failed"); }
+        for (size_t i = 0; i < order.size(); ++i) {
+            const Tile& T = Ts[(size_t)order[i]];
+            const LayerDesc& L = Ls[(size_t)T.layer];
+            TileJob& J = jobs[i];
+            J.tile = order[i]; J.layer = T.layer; J.block0 = T.block0; J.nblocks = T.nblocks; J.bits = L.bits; J.pad_ = 0;
+            J.size = L.size; J.elem_off = L.elem_off; J.word_off = L.word_off; J.block_off = L.block_off; J.pad2_ = 0;
+        }
+        e = cudaMemcpy(p->d_jobs, jobs.data(), jobs.size() * sizeof(TileJob), cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_stage, lev);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->d_levels_enc[0], lev);
@@ -277,7 +286,6 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.lut, nl * kLutEntries);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.ld, nl * kMaxLevels);
     if (e == cudaSuccess) e = dev_alloc_zero(&p->search.fast, nl);
-    if (e == cudaSuccess) e = dev_alloc_zero(&p->search.first, nl);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.norm_partial, KT * (size_t)d.sub_tiles);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.stat_partial, KT);
     if (e == cudaSuccess) e = dev_alloc_zero(&d.sq_diff, KL);
@@ -320,7 +328,7 @@ int lq_plan_create(lq_plan** out, int32_t num_layers, const int64_t* layer_sizes
         free_plan(p);
         return fail(code, "plan setup: %s", cudaGetErrorString(e));
     }
-    d.layers = p->d_layers; d.tiles = p->d_tiles; d.tile_order = p->d_tile_order;
+    d.layers = p->d_layers; d.tiles = p->d_tiles; d.jobs = p->d_jobs;
     e = launch_build_search(d, p->d_levels_enc[0], p->search, nullptr);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -40,6 +40,23 @@ struct Tile {
     int32_t pad_;
 };
 
+// What an encoder CTA needs to know about its tile, one record per CTA in launch order (read with one round trip
+// instead of the chain launch order -> tile -> layer).
+struct TileJob {
+    int32_t tile;         // index in the tile table (the per-tile partials are kept by it)
+    int32_t layer;
+    int32_t block0;       // first block of the tile inside its layer
+    int32_t nblocks;      // 1..kTileBlocks
+    int32_t bits;         // b_m
+    int32_t pad_;
+    int64_t size;         // d_m
+    int64_t elem_off;     // first coordinate of the layer inside a worker's row of `grads`
+    int64_t word_off;     // first word of the layer inside a worker's message
+    int64_t block_off;    // first block of the layer in a worker's row of the zero-row masks
+    int64_t pad2_;
+};
+static_assert(sizeof(TileJob) == 64, "TileJob is read as four 16-byte words");
+
 struct QodaScalars {
     double S;             // running sum of Eq. (general_stepsize)
     double last_delta;    // the term added by the last qoda_step
@@ -56,8 +73,9 @@ struct QodaScalars {
 struct PlanDev {
     const LayerDesc* layers;
     const Tile* tiles;
-    const int32_t* tile_order;   // the order in which the encoder's CTAs take the tiles: all layers advance together, so
-                                 // that layers of different character (dense, mostly zero rows) share the SMs at any time
+    const TileJob* jobs;         // the encoder's tiles in the order in which its CTAs take them: all layers advance
+                                 // together, so that layers of different character (dense, mostly zero rows) share the
+                                 // SMs at any time
     int32_t num_layers;
     int32_t num_tiles;
     int32_t num_workers;
@@ -102,7 +120,6 @@ struct SearchTables {
     uint32_t* lut;     // [L][kLutEntries] per bin: 8 * tau0 | (low 19 bits of the level inside the bin, minus 1) << 13
     float2* ld;        // [L][kMaxLevels]  {l_tau, l_{tau+1} - l_tau}
     int32_t* fast;     // [L]              1 if every bin holds at most one level
-    int32_t* first;    // [L]              first bin whose entry differs from that of bin 0 (the bins below hold no level)
 };
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s);
 cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,

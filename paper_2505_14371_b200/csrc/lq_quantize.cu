@@ -201,37 +201,75 @@ __global__ void __launch_bounds__(kQThreads, 4) quantize_pack_kernel(
     extern __shared__ unsigned char dyn_smem[];
     uint32_t base;
     unsigned char* sm = table_base(dyn_smem, base);
-    const int tile_id = p.tile_order[blockIdx.x];
-    const Tile tile = p.tiles[tile_id];
-    const int layer = tile.layer;
-    const LayerDesc L = p.layers[layer];
-    const int k = blockIdx.y + p.worker0;
+    // CTAs start in the order of their flat index: the workers of one tile next to each other, tiles in the plan's
+    // launch order, so that the last CTAs to start are every worker's short tiles (the ends of the layers) and not
+    // one worker's whole message
+    const int flat = blockIdx.y * gridDim.x + blockIdx.x;
+    const int slot = flat / (int)gridDim.y, kk = flat - slot * (int)gridDim.y;
+    const TileJob J = p.jobs[slot];
+    const int tile_id = J.tile, layer = J.layer;
+    Tile tile;
+    tile.layer = J.layer; tile.block0 = J.block0; tile.nblocks = J.nblocks; tile.pad_ = 0;
+    LayerDesc L;
+    L.elem_off = J.elem_off; L.word_off = J.word_off; L.size = J.size; L.bits = J.bits; L.nlevels = 1 << J.bits;
+    L.block_off = J.block_off;
+    const int k = kk + p.worker0;
     const int lane = threadIdx.x & 31;
     const int64_t kl = (int64_t)k * p.num_layers + layer;
+
+    // Everything below depends on the job record only, so all of it is requested at once: the norms, this thread's
+    // two pieces of the search table, the zero-row masks of its block, the levels of its table entries.
     const float ncur = norms[kl];
     const float nprev = prev_norms ? prev_norms[kl] : 0.0f;
+    const float rn = p.rnorm[kl];
     const bool fast = st.fast[layer] != 0;
-
-    fill_tables(sm, st, layer, L.nlevels, fast, levels_cur, levels_prev, ncur, nprev, kHist);
-    uint8_t* rows_cur = sm + kSmRows;
-    uint8_t* rows_prev = rows_cur + kTileBlocks;
+    const uint4* lsrc = reinterpret_cast<const uint4*>(st.lut + (int64_t)layer * kLutEntries);
+    const uint4 lut0 = __ldg(lsrc + threadIdx.x), lut1 = __ldg(lsrc + kQThreads + threadIdx.x);
+    uint32_t mcur = 0, mprev = 0;
     if (threadIdx.x < tile.nblocks) {
         // a previous message whose masks are unknown is taken as nonzero everywhere
         const int64_t mb = (int64_t)k * p.total_blocks + L.block_off + tile.block0 + threadIdx.x;
-        rows_cur[threadIdx.x] = p.row_mask[mb];
-        rows_prev[threadIdx.x] = (!kStat || !prev_packed) ? (uint8_t)0
-                                 : (p.row_mask_prev ? p.row_mask_prev[mb] : (uint8_t)0xff);
+        mcur = p.row_mask[mb];
+        mprev = (!kStat || !prev_packed) ? 0u : (p.row_mask_prev ? (uint32_t)p.row_mask_prev[mb] : 0xffu);
+    }
+    float lc = 0.f, lp = 0.f;
+    float2 lg = make_float2(0.f, 0.f);
+    if (threadIdx.x < L.nlevels) {
+        lc = levels_cur[(int64_t)layer * kLevelStride + threadIdx.x];
+        lp = levels_prev[(int64_t)layer * kLevelStride + threadIdx.x];
+        lg = st.ld[(int64_t)layer * kMaxLevels + threadIdx.x];
+    }
+    {
+        uint4* ldst = reinterpret_cast<uint4*>(sm + kSmLut);
+        ldst[threadIdx.x] = lut0;
+        ldst[kQThreads + threadIdx.x] = lut1;
+        if (threadIdx.x < L.nlevels) {
+            const float cv = __fmul_rn(ncur, lc), pv = __fmul_rn(nprev, lp);
+            reinterpret_cast<float2*>(sm + kSmLd)[threadIdx.x] = lg;
+            reinterpret_cast<float2*>(sm + kSmTcur)[threadIdx.x] = make_float2(cv, -cv);
+            reinterpret_cast<float2*>(sm + kSmTprev)[threadIdx.x] = make_float2(pv, -pv);
+        }
+        if (kHist) {
+            uint32_t* h = reinterpret_cast<uint32_t*>(sm + kSmHist);
+            for (int i = threadIdx.x; i < LQ_HIST_STRIDE; i += kQThreads) h[i] = 0;
+        }
+    }
+    uint8_t* rows_cur = sm + kSmRows;
+    uint8_t* rows_prev = rows_cur + kTileBlocks;
+    if (threadIdx.x < tile.nblocks) {
+        rows_cur[threadIdx.x] = (uint8_t)mcur;
+        rows_prev[threadIdx.x] = (uint8_t)mprev;
     }
     __syncthreads();
 
     WarpCtx c;
-    c.g = grads + (int64_t)blockIdx.y * p.padded_elems + L.elem_off;
+    c.g = grads + (int64_t)kk * p.padded_elems + L.elem_off;
     c.size = L.size;
     c.nfull = L.size / kBlockCoords;
     c.lane = lane;
     QuantEnv ev;
     ev.lut = base + kSmLut; ev.ld = base + kSmLd; ev.tprev = base + kSmTprev;
-    ev.r = p.rnorm[kl];
+    ev.r = rn;
     ev.hist = reinterpret_cast<uint32_t*>(sm + kSmHist);
     const bool zeroed = ev.r == 0.0f;
     if (step == LQ_STEP_AUTO) step = (uint32_t)p.scalars->t;      // the plan's own iteration counter (graph replays)
@@ -289,15 +327,14 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 //              tau0 = last level (<= n-2) at or below lo; code = (low 19 bits of l_{tau0+1}) - 1 if that level
 //              (<= n-2) lies inside the bin, else all ones, so that  (bits(u) << 13) > lut[bin]  iff  u >= l_{tau0+1}
 //   fast     = no bin holds two or more levels (then tau is tau0 or tau0 + 1)
-//   first    = the first bin whose entry is not bin 0's (tau0 = 0, no level inside)
 __global__ void __launch_bounds__(256) build_search_kernel(PlanDev p, const float* __restrict__ levels,
                                                            SearchTables t)
 {
     __shared__ float lev[kMaxLevels];
-    __shared__ int slow, first;
+    __shared__ int slow;
     const int m = blockIdx.x;
     const int n = p.layers[m].nlevels;
-    if (threadIdx.x == 0) { slow = 0; first = kLutEntries; }
+    if (threadIdx.x == 0) slow = 0;
     for (int i = threadIdx.x; i < n; i += blockDim.x) lev[i] = levels[(int64_t)m * kLevelStride + i];
     __syncthreads();
     for (int i = threadIdx.x; i < kMaxLevels; i += blockDim.x) {
@@ -322,10 +359,9 @@ __global__ void __launch_bounds__(256) build_search_kernel(PlanDev p, const floa
         }
         const uint32_t entry = (code << 13) | (8u * (uint32_t)tau0);
         t.lut[(int64_t)m * kLutEntries + bin] = entry;
-        if (entry != (0x7ffffu << 13)) atomicMin(&first, bin);
     }
     __syncthreads();
-    if (threadIdx.x == 0) { t.fast[m] = slow ? 0 : 1; t.first[m] = first; }
+    if (threadIdx.x == 0) t.fast[m] = slow ? 0 : 1;
 }
 
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s)

@@ -284,13 +284,9 @@ __device__ __forceinline__ void fill_tables(unsigned char* sm, const SearchTable
         tprev[2 * i] = q; tprev[2 * i + 1] = -q;
     }
     if (fast) {
-        // the bins below the first level all hold bin 0's entry (tau0 = 0, no level inside): only the rest is read
         const uint4* src = reinterpret_cast<const uint4*>(st.lut + (int64_t)layer * kLutEntries);
         uint4* dst = reinterpret_cast<uint4*>(sm + kSmLut);
-        const int first4 = st.first[layer] >> 2;
-        const uint32_t e0 = 0x7ffffu << 13;
-        for (int i = threadIdx.x; i < kLutEntries / 4; i += blockDim.x)
-            dst[i] = i < first4 ? make_uint4(e0, e0, e0, e0) : __ldg(src + i);
+        for (int i = threadIdx.x; i < kLutEntries / 4; i += blockDim.x) dst[i] = __ldg(src + i);
     }
     if (hist) {
         uint32_t* h = reinterpret_cast<uint32_t*>(sm + kSmHist);
