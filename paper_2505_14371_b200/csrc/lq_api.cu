@@ -10,7 +10,7 @@
 #include <new>
 #include <vector>
 
-#include "lq_internal.cuh"
+#include "lq_coding.cuh"
 
 using namespace lq;
 
@@ -83,7 +83,7 @@ struct lq_plan {
     int32_t* d_member_layer = nullptr;
     std::vector<int32_t> h_members;        // host staging of both lists (kept alive for the asynchronous copy)
     uint32_t* d_code_enc = nullptr;        // [L][256]   entropy stage, allocated at its first use
-    uint16_t* d_code_dec = nullptr;        // [L][4096]
+    uint16_t* d_code_dec = nullptr;        // [L][kDecEntries]
     uint32_t* d_code_bad = nullptr;        // [1] set by a decode that met an invalid stream
     std::vector<uint8_t> code_len;         // [L][256] host copy of the word lengths
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
@@ -768,13 +768,13 @@ namespace {
 int upload_code(lq_plan* plan, int layer, const uint8_t* len, int n)
 {
     std::vector<uint32_t> code(kMaxLevels, 0), enc(kMaxLevels, 0);
-    std::vector<uint16_t> dec((size_t)1 << kCodeMaxLen);
+    std::vector<uint16_t> dec((size_t)kDecEntries);
     if (!canonical_codes_host(len, n, kCodeMaxLen, code.data()))
         return fail(LQ_EINVAL, "layer %d: lengths must lie in [1, %d] and satisfy Kraft's inequality", layer, kCodeMaxLen);
     build_code_tables_host(len, code.data(), n, enc.data(), dec.data());
     LQ_CUDA(cudaMemcpy(plan->d_code_enc + (size_t)layer * kMaxLevels, enc.data(), kMaxLevels * sizeof(uint32_t),
                        cudaMemcpyHostToDevice));
-    LQ_CUDA(cudaMemcpy(plan->d_code_dec + ((size_t)layer << kCodeMaxLen), dec.data(), dec.size() * sizeof(uint16_t),
+    LQ_CUDA(cudaMemcpy(plan->d_code_dec + (size_t)layer * kDecEntries, dec.data(), dec.size() * sizeof(uint16_t),
                        cudaMemcpyHostToDevice));
     std::copy(len, len + n, plan->code_len.begin() + (size_t)layer * kMaxLevels);
     return LQ_OK;
@@ -787,7 +787,7 @@ int ensure_codes(lq_plan* plan)
     const size_t L = (size_t)(plan->dev.num_layers ? plan->dev.num_layers : 1);
     LQ_CUDA(cudaDeviceSynchronize());
     LQ_CUDA(dev_alloc_zero(&plan->d_code_enc, L * kMaxLevels));
-    LQ_CUDA(dev_alloc_zero(&plan->d_code_dec, L << kCodeMaxLen));
+    LQ_CUDA(dev_alloc_zero(&plan->d_code_dec, L * (size_t)kDecEntries));
     LQ_CUDA(dev_alloc_zero(&plan->d_code_bad, 1));
     try { plan->code_len.assign(L * kMaxLevels, 0); } catch (const std::bad_alloc&) { return fail(LQ_ENOMEM, "host allocation failed"); }
     for (int m = 0; m < plan->dev.num_layers; ++m) {

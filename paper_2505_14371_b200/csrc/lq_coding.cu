@@ -14,7 +14,7 @@
 #include <algorithm>
 #include <vector>
 
-#include "lq_internal.cuh"
+#include "lq_coding.cuh"
 
 namespace lq {
 
@@ -80,18 +80,19 @@ static uint32_t reverse_bits(uint32_t v, int l)
     return r;
 }
 
-// enc[sym] = word with its first bit in bit 0 | length << 16.  dec[next kCodeMaxLen stream bits] = symbol |
-// length << 8, or 0xffff where no word matches (incomplete codes).
+// enc[level] = word with its first bit in bit 0 | length << 16.  dec: the table of lq_coding.cuh.
 void build_code_tables_host(const uint8_t* len, const uint32_t* code, int n, uint32_t* enc, uint16_t* dec)
 {
     for (int i = 0; i < kMaxLevels; ++i) enc[i] = 0;
-    for (int i = 0; i < (1 << kCodeMaxLen); ++i) dec[i] = 0xffffu;
+    for (int i = 0; i < kDecEntries; ++i) dec[i] = (uint16_t)(kDecInvalid | (1u << kDecLenShift));
     for (int s = 0; s < n; ++s) {
         const int l = len[s];
         const uint32_t rev = reverse_bits(code[s], l);
         enc[s] = rev | ((uint32_t)l << 16);
-        for (uint32_t hi = 0; hi < ((uint32_t)1 << (kCodeMaxLen - l)); ++hi)
-            dec[rev | (hi << l)] = (uint16_t)(s | (l << 8));
+        for (uint32_t hi = 0; hi < ((uint32_t)1 << (kDecBits - l)); ++hi) {
+            const uint32_t sign = s != 0 ? (hi & 1u) : 0u;             // the bit right after the word
+            dec[rev | (hi << l)] = (uint16_t)((2u * (uint32_t)s + sign) | ((uint32_t)(l + (s != 0 ? 1 : 0)) << kDecLenShift));
+        }
     }
 }
 
@@ -221,7 +222,7 @@ __global__ void __launch_bounds__(128) entropy_decode_kernel(PlanDev p, const ui
     const LayerDesc L = p.layers[layer];
     const int64_t blk = g - L.block_off;
     const int C = L.bits + 1;
-    const uint16_t* dec = dec_tables + (int64_t)layer * (1 << kCodeMaxLen);
+    const uint16_t* dec = dec_tables + (int64_t)layer * kDecEntries;
     const uint32_t* off_k = offsets + (int64_t)k * (p.total_blocks + 1);
     const int64_t first = off_k[g], last = min((int64_t)off_k[g + 1], capacity);
     const uint32_t* src = in + (int64_t)k * capacity;
@@ -235,12 +236,10 @@ __global__ void __launch_bounds__(128) entropy_decode_kernel(PlanDev p, const ui
         for (int pp = 0; pp < 32; ++pp) {
             if (!real_coord(blk, lane, pp, L.size)) continue;
             while (have <= 32) { const uint32_t x = wi < last ? src[wi] : 0u; ++wi; window |= (uint64_t)x << have; have += 32; }
-            const uint32_t e = dec[window & ((1u << kCodeMaxLen) - 1u)];
-            if (e == 0xffffu) { broken = true; continue; }
-            const uint32_t idx = e & 0xffu, l = e >> 8;
+            const uint32_t e = dec[window & (uint32_t)(kDecEntries - 1)];
+            if (e & kDecInvalid) { broken = true; continue; }
+            const uint32_t sym = e & 0x1ffu, l = e >> kDecLenShift;
             window >>= l; have -= (int)l;
-            uint32_t sym = idx << 1;
-            if (idx != 0u) { sym |= (uint32_t)(window & 1u); window >>= 1; have -= 1; }
             const int off = pp * C, i = off >> 5, s = off & 31;
             cw[i] |= sym << s;
             if (s + C > 32) cw[i + 1] |= sym >> (32 - s);
@@ -250,45 +249,35 @@ __global__ void __launch_bounds__(128) entropy_decode_kernel(PlanDev p, const ui
     if (broken || wi - 2 > last) atomicOr(bad, 1u);           // no valid word, or the block ran past its end
 }
 
-// One thread per run of four lanes (128 coordinates) of a block, eight threads per block, one CTA per sub-tile
-// (32 blocks of one layer): every thread starts at its run's recorded bit offset and rebuilds its four lanes' words.
-// The decode table of the layer sits in shared memory.  A thread that meets no valid word, that would read past
-// the block's end, or that does not end where the next run starts reports a broken stream; nothing is read or
-// written out of bounds.
-template <int C>
-__device__ __forceinline__ void decode_run(const uint32_t* __restrict__ src, int64_t first, int64_t last, uint32_t start_bit,
-                                           uint32_t end_bit, bool check_end, const uint16_t* dec, int64_t blk, int run,
-                                           int64_t size, uint32_t* __restrict__ dst, bool& broken)
+// Decoder on the run offsets.  A run is four lanes (128 coordinates) of a block; one CTA takes a sub-tile (32 blocks
+// of one layer = 256 runs) with the layer's decode table in shared memory.  First every thread looks at one run: a
+// run of 128 zero bits where "0" is the word of level 0 (what untouched rows turn into) is written as zeros at once;
+// the other runs are collected in a list, so that the walk below is done by full warps and not by the few lanes of
+// every warp whose run happens to hold values.  Then thread i walks the i-th run of the list from its recorded bit
+// offset: the next 13 stream bits come from a funnel shift over two of three words kept in registers, one table
+// lookup gives the symbol and the bits taken (the words are refilled every second coordinate).  A run that meets no
+// valid word, that would read past the block's end, or that does not end where the next run starts reports a broken
+// stream; nothing is read or written out of bounds.
+struct RunRef {
+    const uint32_t* src;     // first word of the block's stream
+    int nwords;              // words of the block that may be read
+    uint32_t start_bit, end_bit;
+    bool check_end;          // the run is followed by another run of the block (end_bit is known)
+};
+
+__device__ __forceinline__ uint32_t stream_word(const RunRef& r, int i) { return i < r.nwords ? __ldg(r.src + i) : 0u; }
+
+template <int C, bool kFull>
+__device__ __forceinline__ bool decode_run(const RunRef& r, const uint16_t* dec, int64_t blk, int run, int64_t size,
+                                           uint32_t* __restrict__ dst)
 {
-    int64_t wi = first + (start_bit >> 5);                    // next word to load
-    uint64_t window = 0;
-    int have = 0;                                             // valid bits in the low end of `window`
-    {
-        const uint32_t x = wi < last ? __ldg(src + wi) : 0u; ++wi;
-        window = (uint64_t)(x >> (start_bit & 31u));
-        have = 32 - (int)(start_bit & 31u);
-    }
-    uint32_t used = start_bit;
-    const bool full = (blk + 1) * kBlockCoords <= size;
-    // A run of 128 one-bit words "0" for level index 0 (what untouched rows turn into when 0 is the most frequent
-    // level): 128 zero bits, recognised without walking them.
-    if (full && check_end && end_bit - start_bit == 128u && dec[0] == (uint16_t)(1u << 8)) {
-        const int sh = (int)(start_bit & 31u);
-        const int64_t w0 = first + (start_bit >> 5);
-        uint32_t any = 0;
-        if (w0 + 4 + (sh ? 1 : 0) <= last) {
-            any = __ldg(src + w0) >> sh;
-#pragma unroll
-            for (int i = 1; i < 4; ++i) any |= __ldg(src + w0 + i);
-            if (sh) any |= __ldg(src + w0 + 4) << (32 - sh);
-            if (any == 0u) {
-                for (int l4 = 0; l4 < 4; ++l4)
-#pragma unroll
-                    for (int i = 0; i < C; ++i) dst[i * 32 + 4 * run + l4] = 0u;
-                return;
-            }
-        }
-    }
+    int wi = (int)(r.start_bit >> 5);
+    uint32_t lo = stream_word(r, wi), hi = stream_word(r, wi + 1), nx = stream_word(r, wi + 2);
+    wi += 3;                                                  // next word to load; `lo` is word wi - 3
+    uint32_t sh = r.start_bit & 31u, flags = 0, win = 0;
+    // Coordinates are taken in pairs: with sh < 32 the 32 bits from the current position lie inside {lo, hi}, and
+    // after the first coordinate (at most 13 bits) they still hold the second one whole.
+#pragma unroll 1
     for (int l4 = 0; l4 < 4; ++l4) {
         const int lane = 4 * run + l4;
         uint32_t cw[C + 1];
@@ -296,22 +285,26 @@ __device__ __forceinline__ void decode_run(const uint32_t* __restrict__ src, int
         for (int i = 0; i <= C; ++i) cw[i] = 0u;
 #pragma unroll
         for (int pp = 0; pp < 32; ++pp) {
-            if (!full && !(blk * kBlockCoords + 128 * (pp >> 2) + 4 * lane + (pp & 3) < size)) continue;
-            if (have <= 32) { const uint32_t x = wi < last ? __ldg(src + wi) : 0u; ++wi; window |= (uint64_t)x << have; have += 32; }
-            const uint32_t e = dec[window & ((1u << kCodeMaxLen) - 1u)];
-            if (e == 0xffffu) { broken = true; continue; }
-            const uint32_t idx = e & 0xffu, l = e >> 8;
-            window >>= l; have -= (int)l; used += l;
-            uint32_t sym = idx << 1;
-            if (idx != 0u) { sym |= (uint32_t)(window & 1u); window >>= 1; have -= 1; used += 1u; }
+            if (!kFull && !(blk * kBlockCoords + 128 * (pp >> 2) + 4 * lane + (pp & 3) < size)) continue;
+            if (kFull ? (pp & 1) == 0 : true) {
+                if (sh >= 32u) { sh -= 32u; lo = hi; hi = nx; nx = stream_word(r, wi); ++wi; }
+                win = __funnelshift_r(lo, hi, sh);           // 32 stream bits from the current position
+            }
+            const uint32_t e = dec[win & (uint32_t)(kDecEntries - 1)];
+            flags |= e;
+            win >>= e >> kDecLenShift;                       // at least 19 bits are left for the pair's second coordinate
+            sh += e >> kDecLenShift;
+            const uint32_t sym = e & 0x1ffu;
             const int off = pp * C, i = off >> 5, s = off & 31;
-            cw[i] |= sym << s;
+            cw[i] += sym << s;                               // the fields do not overlap: a multiply-add
             if (s + C > 32) cw[i + 1] |= sym >> (32 - s);
         }
 #pragma unroll
         for (int i = 0; i < C; ++i) dst[i * 32 + lane] = cw[i];
     }
-    if (check_end ? used != end_bit : ((int64_t)((used + 31u) >> 5) > last - first)) broken = true;
+    if (sh >= 32u) { sh -= 32u; ++wi; }                      // (what the next pair's refill would have done)
+    const uint32_t used = 32u * (uint32_t)(wi - 3) + sh;
+    return (flags & kDecInvalid) != 0u || (r.check_end ? used != r.end_bit : used > 32u * (uint32_t)r.nwords);
 }
 
 __global__ void __launch_bounds__(kThreads) entropy_decode_runs_kernel(PlanDev p, const uint32_t* __restrict__ in, int64_t capacity,
@@ -320,36 +313,90 @@ __global__ void __launch_bounds__(kThreads) entropy_decode_runs_kernel(PlanDev p
                                                                        const uint16_t* __restrict__ dec_tables,
                                                                        uint32_t* __restrict__ packed, uint32_t* __restrict__ bad)
 {
-    __shared__ uint16_t dec[1 << kCodeMaxLen];
+    __shared__ __align__(16) uint16_t dec[kDecEntries];
+    __shared__ uint8_t todo[kSubBlocks * LQ_CODE_RUNS];
+    __shared__ int ntodo;
+    static_assert(kSubBlocks * LQ_CODE_RUNS == kThreads, "one thread per run of a sub-tile");
     const Tile tile = p.tiles[blockIdx.x >> p.sub_shift];
     const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
     if (sub0 >= tile.nblocks) return;
     const int layer = tile.layer, k = blockIdx.y;
     const LayerDesc L = p.layers[layer];
     {
-        const uint4* src = reinterpret_cast<const uint4*>(dec_tables + ((int64_t)layer << kCodeMaxLen));
+        const uint4* src = reinterpret_cast<const uint4*>(dec_tables + (int64_t)layer * kDecEntries);
         uint4* dst = reinterpret_cast<uint4*>(dec);
-        for (int i = threadIdx.x; i < (1 << kCodeMaxLen) / 8; i += blockDim.x) dst[i] = __ldg(src + i);
+        for (int i = threadIdx.x; i < kDecEntries / 8; i += blockDim.x) dst[i] = __ldg(src + i);
+    }
+    if (threadIdx.x == 0) ntodo = 0;
+    const int C = L.bits + 1;
+    const uint32_t* off_k = offsets + (int64_t)k * (p.total_blocks + 1);
+    const uint32_t* stream = in + (int64_t)k * capacity;
+    uint32_t* msg = packed + (int64_t)k * p.packed_words + L.word_off;
+    // the run with index t of this sub-tile: block sub0 + t / 8, run t % 8
+    auto run_ref = [&](int t, int64_t& blk) {
+        blk = tile.block0 + sub0 + (t >> 3);
+        const int64_t g = L.block_off + blk;
+        const int64_t first = off_k[g], last = min((int64_t)off_k[g + 1], capacity);
+        const uint16_t* ro = run_offsets + ((int64_t)k * p.total_blocks + g) * LQ_CODE_RUNS;
+        const int run = t & 7;
+        RunRef r;
+        r.src = stream + first;
+        r.nwords = (int)max((int64_t)0, last - first);
+        r.start_bit = ro[run];
+        r.check_end = run + 1 < LQ_CODE_RUNS;
+        r.end_bit = r.check_end ? (uint32_t)ro[run + 1] : 0u;
+        return r;
+    };
+    __syncthreads();
+
+    bool broken = false, walk = false;
+    if (sub0 + (threadIdx.x >> 3) < tile.nblocks) {
+        int64_t blk;
+        const RunRef r = run_ref(threadIdx.x, blk);
+        uint32_t* dst = msg + blk * (int64_t)C * 32;
+        const int run = threadIdx.x & 7;
+        walk = true;
+        if ((int64_t)(r.start_bit >> 5) > (int64_t)r.nwords) {            // an offset that points past the block's end:
+            broken = true; walk = false;                                 // the run's words are still written (zeros)
+            for (int i = 0; i < C; ++i) *reinterpret_cast<uint4*>(dst + i * 32 + 4 * run) = make_uint4(0u, 0u, 0u, 0u);
+        } else if ((blk + 1) * kBlockCoords <= L.size && dec[0] == (uint16_t)kDecZeroBit) {
+            // 128 coordinates of level 0 are 128 zero bits; the last run of a block is followed by zero padding
+            // up to the block's last word
+            const uint32_t nbits = r.check_end ? r.end_bit - r.start_bit : 32u * (uint32_t)r.nwords - r.start_bit;
+            if (r.check_end ? nbits == 128u : (nbits >= 128u && nbits < 160u)) {
+                const uint32_t end = r.start_bit + nbits;
+                const int w0 = (int)(r.start_bit >> 5), w1 = (int)(end >> 5);
+                uint32_t any = stream_word(r, w0) >> (r.start_bit & 31u);
+#pragma unroll
+                for (int i = 1; i < 6; ++i) {
+                    const uint32_t x = stream_word(r, w0 + i);
+                    if (w0 + i < w1) any |= x;
+                    else if (w0 + i == w1 && (end & 31u)) any |= x << (32u - (end & 31u));
+                }
+                if (any == 0u) {
+                    walk = false;
+                    for (int i = 0; i < C; ++i) *reinterpret_cast<uint4*>(dst + i * 32 + 4 * run) = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+        }
+    }
+    {
+        const uint32_t m = __ballot_sync(0xffffffffu, walk);
+        int at = 0;
+        if ((threadIdx.x & 31) == 0 && m) at = atomicAdd(&ntodo, __popc(m));
+        at = __shfl_sync(0xffffffffu, at, 0);
+        if (walk) todo[at + __popc(m & ((1u << (threadIdx.x & 31)) - 1u))] = (uint8_t)threadIdx.x;
     }
     __syncthreads();
-    const int b = sub0 + (threadIdx.x >> 3), run = threadIdx.x & 7;
-    if (b >= tile.nblocks) return;
-    const int64_t blk = tile.block0 + b, g = L.block_off + blk;
-    const uint32_t* off_k = offsets + (int64_t)k * (p.total_blocks + 1);
-    const int64_t first = off_k[g], last = min((int64_t)off_k[g + 1], capacity);
-    const uint16_t* ro = run_offsets + ((int64_t)k * p.total_blocks + g) * LQ_CODE_RUNS;
-    const uint32_t start_bit = ro[run];
-    const uint32_t end_bit = run + 1 < LQ_CODE_RUNS ? (uint32_t)ro[run + 1] : 0u;
-    const int C = L.bits + 1;
-    uint32_t* dst = packed + (int64_t)k * p.packed_words + L.word_off + blk * (int64_t)C * 32;
-    const uint32_t* src = in + (int64_t)k * capacity;
-    bool broken = first + (start_bit >> 5) > last;            // an offset that points past the block's end
-    if (broken) {                                             // the run's words are still written (zeros), nothing is read
-        for (int l4 = 0; l4 < 4; ++l4)
-            for (int i = 0; i < C; ++i) dst[i * 32 + 4 * run + l4] = 0u;
-    } else {
-        switch (C) {
-#define LQ_CASE(CC) case CC: decode_run<CC>(src, first, last, start_bit, end_bit, run + 1 < LQ_CODE_RUNS, dec, blk, run, L.size, dst, broken); break;
+    if ((int)threadIdx.x < ntodo) {
+        const int t = todo[threadIdx.x];
+        int64_t blk;
+        const RunRef r = run_ref(t, blk);
+        uint32_t* dst = msg + blk * (int64_t)C * 32;
+        const bool full = (blk + 1) * kBlockCoords <= L.size;
+        switch (full ? C : -C) {
+#define LQ_CASE(CC) case CC:  broken |= decode_run<CC, true>(r, dec, blk, t & 7, L.size, dst); break;  \
+                    case -CC: broken |= decode_run<CC, false>(r, dec, blk, t & 7, L.size, dst); break;
             LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8) LQ_CASE(9)
 #undef LQ_CASE
             default: break;
