@@ -275,11 +275,13 @@ int lq_symbol_counts(const lq_plan* plan, const uint32_t* packed, uint32_t* coun
  *                   the bit offsets inside the block's stream at which its LQ_CODE_RUNS = 8 runs of 128 coordinates
  *                   (four lanes) start: side data of 16 bytes per block (1/8 bit per coordinate) that is not part of
  *                   the stream and lets the decoder work on the eight runs of a block in parallel.
+ *                   The call uses scratch that the plan allocates at the first use of the stage (64 bytes per block
+ *                   and worker): two encodes of one plan must not overlap on the GPU.
  *   lq_entropy_decode: the inverse, packed fully overwritten; it equals the encoded message except that the sign
  *                   bit of a coordinate with level index 0 comes back as 0 (the stream carries no sign there; the
  *                   decoded value is zero either way).  With run_offsets (as written by lq_entropy_encode for this
- *                   stream) one thread decodes each run, eight per block; with NULL one thread walks a whole block
- *                   (an order of magnitude slower).  A stream with no valid word, a block that runs past its end,
+ *                   stream) one thread decodes each run of 128 coordinates, and runs of untouched rows are not
+ *                   walked; with NULL one thread walks a whole block (an order of magnitude slower).  A stream with no valid word, a block that runs past its end,
  *                   or a run that does not end where the next one starts, sets a flag that lq_entropy_status
  *                   returns (and clears); nothing faults. */
 #define LQ_CODE_MAX_LEN 12

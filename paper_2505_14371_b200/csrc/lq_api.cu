@@ -85,6 +85,7 @@ struct lq_plan {
     uint32_t* d_code_enc = nullptr;        // [L][256]   entropy stage, allocated at its first use
     uint16_t* d_code_dec = nullptr;        // [L][kDecEntries]
     uint32_t* d_code_bad = nullptr;        // [1] set by a decode that met an invalid stream
+    EncodeScratch code_scratch{nullptr, nullptr};   // allocated with the tables
     std::vector<uint8_t> code_len;         // [L][256] host copy of the word lengths
     double alt_qhat = 0.0;         // > 0: qoda_step follows Eq. (Alt) with this exponent
     double* xsum = nullptr;        // caller-owned running sum of the half iterates (qoda_set_average), or NULL
@@ -109,7 +110,7 @@ void free_plan(lq_plan* p)
     cudaFree(p->d_levels_stage); cudaFree(p->d_levels_enc[0]); cudaFree(p->d_levels_enc[1]);
     cudaFree(p->search.lut); cudaFree(p->search.ld); cudaFree(p->search.fast);
     cudaFree(p->dev.norm_partial); cudaFree(p->dev.stat_partial); cudaFree(p->dev.sq_diff);
-    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
+    cudaFree(p->dev.rnorm); cudaFree(p->dev.status); cudaFree(p->dev.scalars); cudaFree(p->d_code_enc); cudaFree(p->d_code_dec); cudaFree(p->d_code_bad); cudaFree(p->code_scratch.lane_bits); cudaFree(p->code_scratch.scan_part); cudaFree(p->d_member_off); cudaFree(p->d_member_layer); cudaFree(p->dev.alt_partial); cudaFree(p->dev.layer_total); cudaFree(p->d_row_mask[0]); cudaFree(p->d_row_mask[1]);
     cudaFree(p->dev.block_live);
     cudaFree(p->dev.energy_partial); cudaFree(p->dev.flag_partial); cudaFree(p->dev.layer_weight);
     for (auto& r : p->prof_recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -789,6 +790,11 @@ int ensure_codes(lq_plan* plan)
     LQ_CUDA(dev_alloc_zero(&plan->d_code_enc, L * kMaxLevels));
     LQ_CUDA(dev_alloc_zero(&plan->d_code_dec, L * (size_t)kDecEntries));
     LQ_CUDA(dev_alloc_zero(&plan->d_code_bad, 1));
+    {
+        const size_t K = (size_t)plan->dev.num_workers, nb = (size_t)(plan->dev.total_blocks ? plan->dev.total_blocks : 1);
+        LQ_CUDA(dev_alloc_zero(&plan->code_scratch.lane_bits, K * nb * 32));
+        LQ_CUDA(dev_alloc_zero(&plan->code_scratch.scan_part, K * ((nb + 1023) / 1024)));
+    }
     try { plan->code_len.assign(L * kMaxLevels, 0); } catch (const std::bad_alloc&) { return fail(LQ_ENOMEM, "host allocation failed"); }
     for (int m = 0; m < plan->dev.num_layers; ++m) {
         const LayerDesc& Ld = plan->layers[(size_t)m];
@@ -870,7 +876,7 @@ int lq_entropy_encode(lq_plan* plan, const uint32_t* packed, uint32_t* stream_wo
     const int rc = ensure_codes(plan);
     if (rc != LQ_OK) return rc;
     LQ_CUDA(launch_entropy_encode(plan->dev, packed, plan->d_code_enc, block_offsets, stream_words, capacity_words,
-                                  run_offsets, (cudaStream_t)stream));
+                                  run_offsets, plan->code_scratch, (cudaStream_t)stream));
     return LQ_OK;
 }
 

@@ -99,14 +99,6 @@ void build_code_tables_host(const uint8_t* len, const uint32_t* code, int n, uin
 // ---- device ------------------------------------------------------------------------------------
 namespace {
 
-// symbol p of a lane's string of 32 symbols of C bits held in C words (C is a run-time value here)
-__device__ __forceinline__ uint32_t symbol_at(const uint32_t* w, int C, int p)
-{
-    const int off = p * C, i = off >> 5, s = off & 31;
-    const uint64_t two = ((uint64_t)w[i + 1] << 32) | w[i];
-    return (uint32_t)(two >> s) & ((1u << C) - 1u);
-}
-
 // Number of real coordinates among the 32 of this lane in block `blk`: coordinate of position p is
 // blk * 1024 + 128 * (p / 4) + 4 * lane + p % 4.
 __device__ __forceinline__ bool real_coord(int64_t blk, int lane, int p, int64_t size)
@@ -114,96 +106,236 @@ __device__ __forceinline__ bool real_coord(int64_t blk, int lane, int p, int64_t
     return blk * kBlockCoords + 128 * (p >> 2) + 4 * lane + (p & 3) < size;
 }
 
-// mode 0: words needed by every block -> sizes[k][block].   mode 1: write the blocks at their offsets.
-template <int kModeWrite>
-__global__ void __launch_bounds__(kThreads) entropy_encode_kernel(PlanDev p, const uint32_t* __restrict__ packed,
-                                                                  const uint32_t* __restrict__ enc_tables,
-                                                                  uint32_t* __restrict__ offsets,
-                                                                  uint32_t* __restrict__ out, int64_t capacity,
-                                                                  uint16_t* __restrict__ run_offsets)
+// symbol p of a lane's string of 32 symbols of C bits held in C words
+template <int C>
+__device__ __forceinline__ uint32_t symbol_at(const uint32_t (&w)[C + 1], int p)
 {
-    __shared__ uint32_t enc[kMaxLevels];
-    __shared__ uint32_t buf[kWarps][1056];
-    Tile tile = p.tiles[blockIdx.x >> p.sub_shift];
-    const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
-    if (sub0 >= tile.nblocks) return;
-    const int sub1 = min(sub0 + kSubBlocks, tile.nblocks);
-    const int layer = tile.layer, k = blockIdx.y;
-    const LayerDesc L = p.layers[layer];
-    const int C = L.bits + 1, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < kMaxLevels; i += blockDim.x) enc[i] = enc_tables[(int64_t)layer * kMaxLevels + i];
-    __syncthreads();
-    const uint32_t* msg = packed + (int64_t)k * p.packed_words + L.word_off;
-    uint32_t* off_k = offsets + (int64_t)k * (p.total_blocks + 1);
-    for (int b = sub0 + warp; b < sub1; b += kWarps) {
-        const int64_t blk = tile.block0 + b;
-        uint32_t w[LQ_MAX_BITS + 2];
-        for (int i = 0; i < C; ++i) w[i] = msg[blk * (int64_t)C * 32 + i * 32 + lane];
+    const int off = p * C, i = off >> 5, s = off & 31;
+    const uint32_t v = s + C <= 32 ? w[i] >> s : __funnelshift_r(w[i], w[i + 1], s);
+    return v & ((1u << C) - 1u);
+}
+
+// Bits that a lane's 32 coordinates take in the stream.  code[symbol] = stream bits of the coordinate (word, then
+// the sign bit of a non-zero level; first bit in bit 0) | their number << 16.
+template <int C, bool kFull>
+__device__ __forceinline__ uint32_t lane_bits(const uint32_t* code, const uint32_t (&w)[C + 1], int64_t blk, int lane,
+                                              int64_t size)
+{
+    uint32_t bits = 0;
+#pragma unroll
+    for (int pp = 0; pp < 32; ++pp) {
+        if (!kFull && !real_coord(blk, lane, pp, size)) continue;
+        bits += code[symbol_at<C>(w, pp)] >> 16;
+    }
+    return bits;
+}
+
+// Writes a lane's coordinates into the block's buffer from bit `pos` on.  The lane's bits gather in {lo, hi} and leave
+// one whole word at a time: the first and the last word it touches may be shared with its neighbours (atomic OR into
+// the zeroed buffer), the words between them are its own (plain stores).
+template <int C, bool kFull>
+__device__ __forceinline__ void lane_emit(const uint32_t* code, const uint32_t (&w)[C + 1], int64_t blk, int lane,
+                                          int64_t size, uint32_t pos, uint32_t* buf)
+{
+    uint32_t lo = 0, hi = 0, f = pos & 31u;
+    uint32_t* dst = buf + (pos >> 5);
+    bool first = true;
+#pragma unroll
+    for (int pp = 0; pp < 32; ++pp) {
+        if (!kFull && !real_coord(blk, lane, pp, size)) continue;
+        const uint32_t e = code[symbol_at<C>(w, pp)], val = e & 0xffffu;
+        lo |= val << f;
+        hi |= __funnelshift_l(val, 0u, f);                    // the bits of val << f above bit 31
+        f += e >> 16;
+        if (f >= 32u) {
+            if (first) atomicOr(dst, lo); else *dst = lo;
+            first = false;
+            ++dst; lo = hi; hi = 0u; f -= 32u;
+        }
+    }
+    if (f) atomicOr(dst, lo);
+}
+
+constexpr int kCodeBufWords = kBlockCoords * (kCodeMaxLen + 1) / 32;      // longest block: every coordinate 13 bits
+
+// What the warps of an encoder CTA share about their sub-tile.
+struct EncodeJob {
+    const uint32_t* msg;         // the layer's words in this worker's message
+    uint32_t* off;               // this worker's block sizes / offsets, at the layer's first block
+    uint32_t* out;               // this worker's stream
+    uint16_t* runs;              // this worker's run offsets at the layer's first block, or NULL
+    uint16_t* lane_bits;         // this worker's bits per lane and block, at the layer's first block
+    int64_t capacity, size;      // words of the stream buffer; coordinates of the layer
+    int block0, block1;          // the sub-tile's blocks [block0, block1) of the layer
+};
+
+// A warp's blocks of a sub-tile for one symbol width (its own function per width, so that each is compiled with
+// its own register budget).  kWrite = false: the words each block needs -> off[block].  true: the blocks are
+// written at off[block].
+template <int C, bool kWrite>
+__device__ __noinline__ void encode_blocks(const EncodeJob& J, const uint32_t* code, uint32_t* bb)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t zero_code = code[0];
+    for (int64_t blk = J.block0 + warp; blk < J.block1; blk += kWarps) {
+        const bool full = (blk + 1) * kBlockCoords <= J.size;
+        uint32_t w[C + 1];
+        uint32_t any = 0;
+#pragma unroll
+        for (int i = 0; i < C; ++i) {
+            w[i] = J.msg[blk * (int64_t)C * 32 + i * 32 + lane];
+            any |= w[i];
+        }
         w[C] = 0u;
-        uint32_t bits = 0;                                   // bits of this lane's 32 coordinates
-        for (int pp = 0; pp < 32; ++pp) {
-            if (!real_coord(blk, lane, pp, L.size)) continue;
-            const uint32_t sym = symbol_at(w, C, pp);
-            bits += (enc[sym >> 1] >> 16) + ((sym >> 1) != 0u ? 1u : 0u);
+        // a lane whose coordinates are all level 0 (untouched rows): 32 times the word of level 0
+        const bool plain = full && any == 0u;
+        uint32_t bits;
+        if (kWrite) bits = J.lane_bits[blk * 32 + lane];     // sized by the first pass
+        else {
+            bits = 32u * (zero_code >> 16);
+            if (!plain) bits = full ? lane_bits<C, true>(code, w, blk, lane, J.size) : lane_bits<C, false>(code, w, blk, lane, J.size);
+            J.lane_bits[blk * 32 + lane] = (uint16_t)bits;
         }
         uint32_t incl = bits;                                // inclusive prefix sum over the lanes
+#pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += t;
         }
         const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
         const uint32_t nwords = (total + 31u) >> 5;
-        if (!kModeWrite) {
-            if (lane == 0) off_k[L.block_off + blk] = nwords;
-            continue;
-        }
-        for (uint32_t i = lane; i < nwords; i += 32) buf[warp][i] = 0u;
+        if constexpr (!kWrite) {
+            if (lane == 0) J.off[blk] = nwords;
+        } else {
+        for (uint32_t i = lane; i < nwords; i += 32) bb[i] = 0u;
         __syncwarp();
-        uint32_t pos = incl - bits;
+        const uint32_t pos = incl - bits;
         // where the runs of four lanes (128 coordinates) start inside the block's stream: lets a decoder work on
         // eight runs of a block at once
-        if (run_offsets && (lane & 3) == 0)
-            run_offsets[((int64_t)k * p.total_blocks + L.block_off + blk) * LQ_CODE_RUNS + (lane >> 2)] = (uint16_t)pos;
-        for (int pp = 0; pp < 32; ++pp) {
-            if (!real_coord(blk, lane, pp, L.size)) continue;
-            const uint32_t sym = symbol_at(w, C, pp), idx = sym >> 1;
-            const uint32_t e = enc[idx], l = e >> 16;
-            uint32_t val = e & 0xffffu, nb = l;
-            if (idx != 0u) { val |= (sym & 1u) << l; nb += 1u; }
-            const uint32_t wi = pos >> 5, sh = pos & 31u;
-            atomicOr(&buf[warp][wi], val << sh);
-            if (sh + nb > 32u) atomicOr(&buf[warp][wi + 1], val >> (32u - sh));
-            pos += nb;
+        if (J.runs && (lane & 3) == 0) J.runs[blk * LQ_CODE_RUNS + (lane >> 2)] = (uint16_t)pos;
+        if (!(plain && (zero_code & 0xffffu) == 0u)) {       // (32 words "0...0" of level 0 are already there)
+            if (full) lane_emit<C, true>(code, w, blk, lane, J.size, pos, bb);
+            else      lane_emit<C, false>(code, w, blk, lane, J.size, pos, bb);
         }
         __syncwarp();
-        const int64_t first = off_k[L.block_off + blk];
-        if (first + nwords <= capacity) {                    // a stream buffer that is too small is never overrun
-            uint32_t* dst = out + (int64_t)k * capacity + first;
-            for (uint32_t i = lane; i < nwords; i += 32) dst[i] = buf[warp][i];
+        const int64_t first = J.off[blk];
+        if (first + nwords <= J.capacity) {                  // a stream buffer that is too small is never overrun
+            for (uint32_t i = lane; i < nwords; i += 32) J.out[first + i] = bb[i];
         }
         __syncwarp();
+        }
     }
 }
 
-// Exclusive prefix sum of each worker's block sizes, in place; entry [blocks] receives the total.
-__global__ void __launch_bounds__(1024) entropy_scan_kernel(PlanDev p, uint32_t* __restrict__ offsets)
+// One warp per block, one CTA per sub-tile (32 blocks of one layer).
+// kModeWrite = 0: words needed by every block -> sizes[k][block].   1: write the blocks at their offsets.
+template <int kModeWrite>
+__global__ void __launch_bounds__(kThreads, 4) entropy_encode_kernel(PlanDev p, const uint32_t* __restrict__ packed,
+                                                                     const uint32_t* __restrict__ enc_tables,
+                                                                     uint32_t* __restrict__ offsets,
+                                                                     uint32_t* __restrict__ out, int64_t capacity,
+                                                                     uint16_t* __restrict__ run_offsets,
+                                                                     uint16_t* __restrict__ lane_bits)
 {
-    __shared__ uint32_t part[1024];
-    uint32_t* a = offsets + (int64_t)blockIdx.x * (p.total_blocks + 1);
-    const int64_t n = p.total_blocks;
-    const int64_t per = (n + 1023) / 1024, lo = threadIdx.x * per, hi = min(n, lo + per);
-    uint32_t sum = 0;
-    for (int64_t i = lo; i < hi; ++i) sum += a[i];
-    part[threadIdx.x] = sum;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t run = 0;
-        for (int i = 0; i < 1024; ++i) { const uint32_t t = part[i]; part[i] = run; run += t; }
-        a[n] = run;
+    __shared__ uint32_t code[2 * kMaxLevels];
+    __shared__ uint32_t buf[kModeWrite ? kWarps : 1][kModeWrite ? kCodeBufWords : 1];
+    Tile tile = p.tiles[blockIdx.x >> p.sub_shift];
+    const int sub0 = (blockIdx.x & (p.sub_tiles - 1)) * kSubBlocks;
+    if (sub0 >= tile.nblocks) return;
+    const int layer = tile.layer, k = blockIdx.y;
+    const LayerDesc L = p.layers[layer];
+    // per symbol (2 * level + sign): the level's word, the sign bit behind it unless the level is 0, and their length
+    for (int sym = threadIdx.x; sym < 2 * L.nlevels; sym += blockDim.x) {
+        const uint32_t e = enc_tables[(int64_t)layer * kMaxLevels + (sym >> 1)], l = e >> 16;
+        code[sym] = (sym >> 1) ? ((e & 0xffffu) | ((uint32_t)(sym & 1) << l) | ((l + 1u) << 16)) : e;
     }
     __syncthreads();
-    uint32_t run = part[threadIdx.x];
-    for (int64_t i = lo; i < hi; ++i) { const uint32_t t = a[i]; a[i] = run; run += t; }
+    EncodeJob J;
+    J.msg = packed + (int64_t)k * p.packed_words + L.word_off;
+    J.off = offsets + (int64_t)k * (p.total_blocks + 1) + L.block_off;
+    J.out = out + (int64_t)k * capacity;
+    J.runs = run_offsets ? run_offsets + ((int64_t)k * p.total_blocks + L.block_off) * LQ_CODE_RUNS : nullptr;
+    J.lane_bits = lane_bits + ((int64_t)k * p.total_blocks + L.block_off) * 32;
+    J.capacity = capacity; J.size = L.size;
+    J.block0 = tile.block0 + sub0; J.block1 = tile.block0 + min(sub0 + kSubBlocks, tile.nblocks);
+    uint32_t* bb = buf[kModeWrite ? (threadIdx.x >> 5) : 0];
+    switch (L.bits + 1) {
+#define LQ_CASE(CC) case CC: encode_blocks<CC, kModeWrite != 0>(J, code, bb); break;
+        LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8) LQ_CASE(9)
+#undef LQ_CASE
+        default: break;
+    }
+}
+
+// Exclusive prefix sum of each worker's block sizes, in place; entry [blocks] receives the total.  Two launches:
+// the sum of every 1024 consecutive sizes, then each CTA adds the sums before its chunk and scans the chunk.
+__global__ void __launch_bounds__(1024) entropy_scan_sums_kernel(PlanDev p, const uint32_t* __restrict__ offsets,
+                                                                 uint32_t* __restrict__ part)
+{
+    __shared__ uint32_t red[32];
+    const uint32_t* a = offsets + (int64_t)blockIdx.y * (p.total_blocks + 1);
+    const int64_t i = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    uint32_t v = i < p.total_blocks ? a[i] : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        v = red[threadIdx.x];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (threadIdx.x == 0) part[(int64_t)blockIdx.y * gridDim.x + blockIdx.x] = v;
+    }
+}
+
+__global__ void __launch_bounds__(1024) entropy_scan_apply_kernel(PlanDev p, uint32_t* __restrict__ offsets,
+                                                                  const uint32_t* __restrict__ part)
+{
+    __shared__ uint32_t red[32];
+    __shared__ uint32_t base_s;
+    uint32_t* a = offsets + (int64_t)blockIdx.y * (p.total_blocks + 1);
+    const uint32_t* pk = part + (int64_t)blockIdx.y * gridDim.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // the sum of the chunks before this one (and, in the last CTA, of all chunks: the stream's length)
+    uint32_t before = 0, all = 0;
+    for (int c = threadIdx.x; c < (int)gridDim.x; c += 1024) {
+        const uint32_t v = pk[c];
+        all += v;
+        if (c < (int)blockIdx.x) before += v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { before += __shfl_xor_sync(0xffffffffu, before, o); all += __shfl_xor_sync(0xffffffffu, all, o); }
+    if (lane == 0) red[warp] = before;
+    __syncthreads();
+    if (threadIdx.x == 0) { uint32_t t = 0; for (int w = 0; w < 32; ++w) t += red[w]; base_s = t; }
+    __syncthreads();
+    if (blockIdx.x == gridDim.x - 1) {
+        if (lane == 0) red[warp] = all;
+        __syncthreads();
+        if (threadIdx.x == 0) { uint32_t t = 0; for (int w = 0; w < 32; ++w) t += red[w]; a[p.total_blocks] = t; }
+    }
+    __syncthreads();
+    const int64_t i = (int64_t)blockIdx.x * 1024 + threadIdx.x;
+    const uint32_t v = i < p.total_blocks ? a[i] : 0u;
+    uint32_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) red[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = red[lane], wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += t;
+        }
+        red[lane] = wi - w;                                  // exclusive over the warps
+    }
+    __syncthreads();
+    if (i < p.total_blocks) a[i] = base_s + red[warp] + incl - v;
 }
 
 // One thread per (block, worker): walks the block's stream and rebuilds the fixed-width words.
@@ -408,13 +540,16 @@ __global__ void __launch_bounds__(kThreads) entropy_decode_runs_kernel(PlanDev p
 }  // namespace
 
 cudaError_t launch_entropy_encode(const PlanDev& p, const uint32_t* packed, const uint32_t* enc_tables,
-                                  uint32_t* offsets, uint32_t* out, int64_t capacity, uint16_t* run_offsets, cudaStream_t s)
+                                  uint32_t* offsets, uint32_t* out, int64_t capacity, uint16_t* run_offsets,
+                                  EncodeScratch scratch, cudaStream_t s)
 {
     if (p.num_tiles == 0) return cudaSuccess;
     const dim3 grid((unsigned)p.num_tiles * p.sub_tiles, (unsigned)p.num_workers);
-    entropy_encode_kernel<0><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, nullptr);
-    entropy_scan_kernel<<<(unsigned)p.num_workers, 1024, 0, s>>>(p, offsets);
-    entropy_encode_kernel<1><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, run_offsets);
+    const dim3 chunks((unsigned)((p.total_blocks + 1023) / 1024), (unsigned)p.num_workers);
+    entropy_encode_kernel<0><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, nullptr, scratch.lane_bits);
+    entropy_scan_sums_kernel<<<chunks, 1024, 0, s>>>(p, offsets, scratch.scan_part);
+    entropy_scan_apply_kernel<<<chunks, 1024, 0, s>>>(p, offsets, scratch.scan_part);
+    entropy_encode_kernel<1><<<grid, kThreads, 0, s>>>(p, packed, enc_tables, offsets, out, capacity, run_offsets, scratch.lane_bits);
     return cudaGetLastError();
 }
 

@@ -141,15 +141,6 @@ cudaError_t launch_decode(const PlanDev& p, const uint32_t* packed, const float*
 cudaError_t launch_level_probabilities(const PlanDev& p, const uint32_t* hist, const float* norms, int num_samples,
                                        const float* levels, double* probs, cudaStream_t s);
 cudaError_t launch_symbol_counts(const PlanDev& p, const uint32_t* packed, uint32_t* counts, cudaStream_t s);
-// entropy stage (lq_coding.cu)
-bool huffman_lengths_host(const double* w, int n, int max_len, uint8_t* len);
-bool canonical_codes_host(const uint8_t* len, int n, int max_len, uint32_t* code);
-void build_code_tables_host(const uint8_t* len, const uint32_t* code, int n, uint32_t* enc, uint16_t* dec);
-cudaError_t launch_entropy_encode(const PlanDev& p, const uint32_t* packed, const uint32_t* enc_tables,
-                                  uint32_t* offsets, uint32_t* out, int64_t capacity, uint16_t* run_offsets, cudaStream_t s);
-cudaError_t launch_entropy_decode(const PlanDev& p, const uint32_t* in, int64_t capacity, const uint32_t* offsets,
-                                  const uint16_t* run_offsets, const uint16_t* dec_tables, uint32_t* packed, uint32_t* bad,
-                                  cudaStream_t s);
 cudaError_t launch_block_live(const PlanDev& p, cudaStream_t s);
 cudaError_t launch_alt_scalars(const PlanDev& p, double qhat, cudaStream_t s);
 cudaError_t launch_alt_finalize(const PlanDev& p, cudaStream_t s);
