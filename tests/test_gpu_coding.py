@@ -131,6 +131,83 @@ def test_stream_matches_the_oracle_and_round_trips(lqm, orc, bits):
     assert np.array_equal(to_unpadded(plan, g1), to_unpadded(plan, g2))              # padding between layers aside
 
 
+@pytest.mark.parametrize("code", ["zero_is_one_bit", "flat", "zero_is_long"])
+def test_untouched_rows_and_blocks(lqm, orc, code):
+    """Messages with untouched rows, untouched blocks and an untouched layer end, under three codes: level 0 sent as
+    the one-bit word "0" (what a fitted code gives it: runs of zero bits, which neither side walks), the flat code
+    (level 0 is b zero bits), and a code whose word for level 0 is long and not all zeros (nothing can be left out).
+    Stream and run offsets against the oracle's encoder block by block, and the round trip with and without the offsets."""
+    bits, K = 3, 2
+    sizes = [7 * 1024 + 300, 4 * 1024, 2048 + 128 * 3 + 5]
+    plan = lqm.Plan(sizes, [bits] * 3, 2, K, SEED + 77)
+    g = torch.Generator(device="cuda").manual_seed(77)
+    grads = torch.randn((K, plan.padded_elems), generator=g, device="cuda") ** 3 * 0.05
+    for k in range(K):
+        for m in range(3):
+            v = grads[k, plan.elem_offsets[m]: plan.elem_offsets[m] + sizes[m]]
+            rows = torch.rand((sizes[m] + 127) // 128, generator=g, device="cuda") < 0.75       # untouched rows of 128
+            v[rows.repeat_interleave(128)[: sizes[m]]] = 0
+        grads[k, plan.elem_offsets[0] + 2048: plan.elem_offsets[0] + 4096] = 0                  # two untouched blocks
+        grads[k, plan.elem_offsets[1]: plan.elem_offsets[1] + 1024 * (1 + k)] = 0
+        grads[k, plan.elem_offsets[2] + 2048: plan.elem_offsets[2] + sizes[2]] = 0              # an untouched partial block
+    packed = plan.empty_packed(); norms = plan.empty_norms()
+    plan.lq_quantize_pack(grads, 1, packed, norms)
+    n = 1 << bits
+    weights = {"zero_is_one_bit": [0.9] + [0.1 / (n - 1)] * (n - 1), "zero_is_long": [0.001, 0.5, 0.25, 0.12, 0.06, 0.03, 0.02, 0.019]}
+    lengths = [bits] * n if code == "flat" else lqm.lq_code_build(weights[code])
+    if code == "zero_is_one_bit":
+        assert lengths[0] == 1
+    if code == "zero_is_long":
+        assert lengths[0] > 3
+    for m in range(3):
+        plan.lq_code_set(m, lengths)
+    runs = plan.empty_run_offsets()
+    cap = plan.lq_plan_blocks() * 416
+    stream = torch.full((K, cap), -1, dtype=torch.int32, device="cuda")
+    offs = torch.zeros((K, plan.lq_plan_blocks() + 1), dtype=torch.int32, device="cuda")
+    plan.lq_entropy_encode(packed, stream, offs, runs)
+    torch.cuda.synchronize()
+    model = oracle_model(orc, plan)
+    ref = model.quantize(to_unpadded(plan, grads), 1)
+    S = stream.cpu().numpy().view(np.uint32); O = offs.cpu().numpy().astype(np.int64); R = runs.cpu().numpy().view(np.uint16)
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    l = np.uint8(lengths); c = orc.canonical_codes(l); l64 = l.astype(np.int64)
+    for k in range(K):
+        gb = 0; pos = 0
+        for m, d in enumerate(sizes):
+            for blk in range((d + 1023) // 1024):
+                lo = off[m] + blk * 1024; hi = min(off[m] + d, lo + 1024)
+                words, _ = orc.entropy_encode_block(ref["idx"][k, lo:hi], ref["sign"][k, lo:hi], l, c)
+                assert O[k, gb] == pos and np.array_equal(S[k, pos: pos + words.size], words), (k, m, blk)
+                ss = np.arange(1024); lane, pp = ss // 32, ss % 32
+                coord = blk * 1024 + 128 * (pp // 4) + 4 * lane + pp % 4
+                real = coord < d
+                ix = np.zeros(1024, np.int64); ix[real] = ref["idx"][k, off[m] + coord[real]]
+                nb = np.where(real, l64[ix] + (ix != 0), 0)
+                assert np.array_equal(R[k, gb].astype(np.int64), np.concatenate([[0], np.cumsum(nb)])[0:1024:128]), (k, m, blk)
+                pos += words.size; gb += 1
+        assert O[k, gb] == pos
+    want = _canonical(orc, plan, packed)
+    for r in (runs, None):
+        back = torch.full_like(packed, -1)
+        plan.lq_entropy_decode(stream, offs, back, r)
+        torch.cuda.synchronize()
+        assert plan.lq_entropy_status() == 0
+        assert np.array_equal(back.cpu().numpy().view(np.uint32), want)
+    # a one in the middle of a run of zero bits is a different message, not an untouched row: with the one-bit word for
+    # level 0 the decoder must not take the run for zeros
+    if code == "zero_is_one_bit":
+        k, gb = 0, 2                                                     # an untouched block of worker 0
+        first = int(O[k, gb])
+        assert np.all(S[k, first: int(O[k, gb + 1])] == 0)
+        broken = stream.clone(); broken[k, first + 1] = 1 << 7
+        back = torch.full_like(packed, -1)
+        plan.lq_entropy_decode(broken, offs, back, runs)
+        torch.cuda.synchronize()
+        got = back.cpu().numpy().view(np.uint32)
+        assert plan.lq_entropy_status() != 0 or not np.array_equal(got, want)
+
+
 def test_fitted_code_beats_the_fixed_width_and_meets_the_entropy_bound(lqm, orc):
     """Codes built from the estimated level probabilities: the stream is shorter than the fixed-width message, and the
     bits spent on level words per coordinate lie between the empirical entropy and the entropy + 1."""
