@@ -41,11 +41,11 @@ KERNEL_SOURCES = {"norm_partial": ["lq_norm.cu", "lq_internal.cuh"],
                   "quantize_pack": ["lq_quantize.cu", "lq_quantize.cuh", "lq_internal.cuh"],
                   "decode": ["lq_decode.cu", "lq_internal.cuh"]}
 NCU_SCALED = {"transformer_xl": {          # kernel: bytes per embedding / other worker-coordinate, warp instr likewise
-    "norm_partial": {"bytes": (4.0098, 4.0070), "inst": (0.15710, 0.16787), "sources": "4529730d911b253d"},
-    "quantize_pack": {"bytes": (1.3164, 5.3338), "inst": (0.22499, 1.29303), "sources": "95997987bbe668a4"},
-    "decode": {"bytes": (2.1174, 2.6349), "inst": (0.23964, 0.24161), "sources": "6b82b169a3f46c71"}}}
+    "norm_partial": {"bytes": (4.0064, 4.0086), "inst": (0.15710, 0.16787), "sources": "d9c88bc1e0cc1e6b"},
+    "quantize_pack": {"bytes": (1.3174, 5.3327), "inst": (0.22499, 1.29303), "sources": "2aea497ea512889b"},
+    "decode": {"bytes": (2.1186, 2.6344), "inst": (0.23964, 0.24161), "sources": "de040b4901edcbaa"}}}
 NCU_DIRECT = {"flat:26:4:8:2": {           # kernel: bytes and warp instructions of one launch
-    "quantize_pack": {"bytes": 2485956096.0 + 354845696.0, "inst": 679542784.0, "sources": "95997987bbe668a4"}}}
+    "quantize_pack": {"bytes": 2485287424.0 + 354692096.0, "inst": 679542784.0, "sources": "2aea497ea512889b"}}}
 DENSE_POINT = "flat:26:4:8:2"             # dense companion of the headline workload: no zero rows to skip
 ISSUE_PEAK = 148 * 4 * 1.965e9            # warp instructions per second: 148 SMs x 4 schedulers x 1 per clock at 1965 MHz
 
