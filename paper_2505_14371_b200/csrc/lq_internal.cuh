@@ -119,7 +119,8 @@ cudaError_t launch_norm_finalize(const PlanDev& p, float* norms, cudaStream_t s)
 struct SearchTables {
     uint32_t* lut;     // [L][kLutEntries] per bin: 8 * tau0 | (low 19 bits of the level inside the bin, minus 1) << 13
     float2* ld;        // [L][kMaxLevels]  {l_tau, l_{tau+1} - l_tau}
-    int32_t* fast;     // [L]              1 if every bin holds at most one level
+    int32_t* fast;     // [L]              1 if every bin holds at most one level; else 1 + R (byte table over the top 15
+                       //                  bits in lut's place, at most R levels per bin)
 };
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s);
 cudaError_t launch_quantize(const PlanDev& p, const float* grads, uint32_t step, uint32_t* packed,

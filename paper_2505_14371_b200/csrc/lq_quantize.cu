@@ -92,7 +92,7 @@ __device__ __noinline__ double quantize_partial_block(const PlanDev& p, const Qu
 // A warp's share of a tile: the whole blocks warp, warp + 8, ...  A block whose rows are all zero in this input
 // and in the input behind the previous message is an all-zero piece of message that adds nothing to the
 // statistic: its words are stored and nothing is read.  The other blocks are taken in order.
-template <int B, bool kFast, bool kHist, bool kStat>
+template <int B, int kSearch, bool kHist, bool kStat>
 __device__ __forceinline__ double quantize_tile(const PlanDev& p, const PhiloxConsts& pc, const WarpCtx& c,
                                                 const Tile& tile, uint32_t* __restrict__ out,
                                                 const uint32_t* __restrict__ prev, const QuantEnv& ev,
@@ -166,7 +166,7 @@ __device__ __forceinline__ double quantize_tile(const PlanDev& p, const PhiloxCo
                 const float vv[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    quantize_coord<B, kFast, kHist, kStat, false>(ev, vv[e], x[e], 4 * j + e, cw, pw, stat, 0.f, 0.f, true);
+                    quantize_coord<B, kSearch, kHist, kStat, false>(ev, vv[e], x[e], 4 * j + e, cw, pw, stat, 0.f, 0.f, true);
             } else {
                 if ((mnext >> j) & 1u) cp_async16(ring + 512u * j, nsrc + 128 * j, 16);
                 cp_async_commit();
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(kQThreads, 4) quantize_pack_kernel(
     const float ncur = norms[kl];
     const float nprev = prev_norms ? prev_norms[kl] : 0.0f;
     const float rn = p.rnorm[kl];
-    const bool fast = st.fast[layer] != 0;
+    const int search = st.fast[layer];                      // 1: one lookup; 1 + R: byte table and up to R steps
     const uint4* lsrc = reinterpret_cast<const uint4*>(st.lut + (int64_t)layer * kLutEntries);
     const uint4 lut0 = __ldg(lsrc + threadIdx.x), lut1 = __ldg(lsrc + kQThreads + threadIdx.x);
     uint32_t mcur = 0, mprev = 0;
@@ -270,6 +270,7 @@ __global__ void __launch_bounds__(kQThreads, 4) quantize_pack_kernel(
     QuantEnv ev;
     ev.lut = base + kSmLut; ev.ld = base + kSmLd; ev.tprev = base + kSmTprev;
     ev.r = rn;
+    ev.refine = search - 1;
     ev.hist = reinterpret_cast<uint32_t*>(sm + kSmHist);
     const bool zeroed = ev.r == 0.0f;
     if (step == LQ_STEP_AUTO) step = (uint32_t)p.scalars->t;      // the plan's own iteration counter (graph replays)
@@ -278,12 +279,12 @@ __global__ void __launch_bounds__(kQThreads, 4) quantize_pack_kernel(
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
 
     double stat = 0.0;
-    switch (zeroed ? -L.bits : L.bits * 2 + (fast ? 1 : 0)) {
+    switch (zeroed ? -L.bits : L.bits * 2 + (search == 1 ? 1 : 0)) {
 #define LQ_CASE(BB)                                                                              \
     case -BB:        stat = kStat ? zeroed_tile<BB>(tile, lane, out, prev, ev.tprev)             \
                                   : zeroed_tile<BB>(tile, lane, out, nullptr, ev.tprev); break;  \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist, kStat>(p, pc, c, tile, out, prev, ev, rows_cur, rows_prev, base + kSmRing); break;  \
-    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist, kStat>(p, pc, c, tile, out, prev, ev, rows_cur, rows_prev, base + kSmRing); break;
+    case 2 * BB:     stat = quantize_tile<BB, 2, kHist, kStat>(p, pc, c, tile, out, prev, ev, rows_cur, rows_prev, base + kSmRing); break;  \
+    case 2 * BB + 1: stat = quantize_tile<BB, 1, kHist, kStat>(p, pc, c, tile, out, prev, ev, rows_cur, rows_prev, base + kSmRing); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;
@@ -326,15 +327,18 @@ __global__ void __launch_bounds__(128) stat_finalize_kernel(PlanDev p)
 //   lut[bin] = 8 * tau0 | code << 13    bin = bits(u) >> 19, i.e. the values [lo, hi) with bits(lo) = bin << 19;
 //              tau0 = last level (<= n-2) at or below lo; code = (low 19 bits of l_{tau0+1}) - 1 if that level
 //              (<= n-2) lies inside the bin, else all ones, so that  (bits(u) << 13) > lut[bin]  iff  u >= l_{tau0+1}
-//   fast     = no bin holds two or more levels (then tau is tau0 or tau0 + 1)
+//   fast     = 1: no bin holds two or more levels (then tau is tau0 or tau0 + 1)
+// Layers with denser levels (8-bit codes) get a byte table over the top 15 bits instead, in the same 8 KB:
+//   lut8[bits(u) >> 17] = tau0 of that finer bin; tau is found by stepping up while l_{tau+1} <= u, at most R times,
+//   R = the most levels inside one bin;  fast = 1 + R.
 __global__ void __launch_bounds__(256) build_search_kernel(PlanDev p, const float* __restrict__ levels,
                                                            SearchTables t)
 {
     __shared__ float lev[kMaxLevels];
-    __shared__ int slow;
+    __shared__ int slow, most;
     const int m = blockIdx.x;
     const int n = p.layers[m].nlevels;
-    if (threadIdx.x == 0) slow = 0;
+    if (threadIdx.x == 0) { slow = 0; most = 0; }
     for (int i = threadIdx.x; i < n; i += blockDim.x) lev[i] = levels[(int64_t)m * kLevelStride + i];
     __syncthreads();
     for (int i = threadIdx.x; i < kMaxLevels; i += blockDim.x) {
@@ -361,7 +365,23 @@ __global__ void __launch_bounds__(256) build_search_kernel(PlanDev p, const floa
         t.lut[(int64_t)m * kLutEntries + bin] = entry;
     }
     __syncthreads();
-    if (threadIdx.x == 0) t.fast[m] = slow ? 0 : 1;
+    if (slow) {
+        uint8_t* lut8 = reinterpret_cast<uint8_t*>(t.lut + (int64_t)m * kLutEntries);
+        for (int bin = threadIdx.x; bin < 4 * kLutEntries; bin += blockDim.x) {
+            const uint32_t lob = (uint32_t)bin << 17;
+            const bool top = lob >= 0x3f800000u;
+            const float lo = __uint_as_float(top ? 0x3f800000u : lob);
+            int tau0 = 0, inside = 0;
+            for (int j = 1; j <= n - 2; ++j) {
+                if (lev[j] <= lo) tau0 = j;
+                else if (!top && (__float_as_uint(lev[j]) >> 17) == (uint32_t)bin) ++inside;
+            }
+            lut8[bin] = (uint8_t)tau0;
+            atomicMax(&most, inside);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) t.fast[m] = slow ? 1 + most : 1;
 }
 
 cudaError_t launch_build_search(const PlanDev& p, const float* levels, SearchTables t, cudaStream_t s)

@@ -51,6 +51,12 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t a)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
+__device__ __forceinline__ uint32_t lds_u8(uint32_t a)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ float lds_f32(uint32_t a)
 {
     float v;
@@ -80,6 +86,12 @@ __device__ __forceinline__ uint32_t add8_if_gt_u32(uint32_t x, uint32_t a, uint3
 __device__ __forceinline__ uint32_t add8_if_lt(uint32_t x, float a, float b)
 {
     asm("{\n\t.reg .pred p;\n\tsetp.lt.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(x) : "f"(a), "f"(b));
+    return x;
+}
+// x + 8 when a <= b, else x
+__device__ __forceinline__ uint32_t add8_if_le(uint32_t x, float a, float b)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.le.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(x) : "f"(a), "f"(b));
     return x;
 }
 // x + 4 when v < 0 (so neither zero sets the sign bit of a symbol), else x
@@ -203,6 +215,8 @@ __device__ __forceinline__ void philox4x32_10_folded(uint32_t ctr0, const Philox
 struct QuantEnv {
     uint32_t lut, ld, tprev;
     float r;
+    int refine;          // layers whose levels are too dense for the one-lookup search: byte table over the top 15
+                         // bits, then up to `refine` steps upwards
     uint32_t* hist;      // the CTA's histogram (generic pointer), histogram mode only
 };
 
@@ -211,7 +225,7 @@ struct QuantEnv {
 // x: the coordinate's Philox word.  Bucket scope: the value tables hold the plain signed levels and the row's
 // norms (nrow now, pn in the previous message) scale them.  `counted`: the coordinate lies inside the layer
 // (histogram mode).
-template <int B, bool kFast, bool kHist, bool kStat, bool kBucket>
+template <int B, int kSearch, bool kHist, bool kStat, bool kBucket>
 __device__ __forceinline__ void quantize_coord(const QuantEnv& ev, float v, uint32_t x, int pp,
                                                uint32_t (&cw)[B + 1], const uint32_t (&pw)[B + 1], double& stat,
                                                float nrow, float pn, bool counted)
@@ -222,17 +236,14 @@ __device__ __forceinline__ void quantize_coord(const QuantEnv& ev, float v, uint
     const float u = __fmul_rn(fabsf(v), ev.r);
     const uint32_t ub = __float_as_uint(u);
     uint32_t t8;                                             // address of {l_tau, gap}
-    if (kFast) {
+    if (kSearch == 1) {
         const uint32_t e = lds_u32(((ub >> 17) & 0x1FFCu) | ev.lut);
         t8 = add8_if_gt_u32((e & 0x7F8u) | ev.ld, ub << 13, e);
     } else {
-        int tau = 0;
-#pragma unroll
-        for (int s = B - 1; s >= 0; --s) {
-            const int cand = tau + (1 << s);
-            if (lds_f32(ev.ld + 8u * (uint32_t)cand) <= u) tau = cand;
-        }
-        t8 = ev.ld + 8u * (uint32_t)min(tau, n - 2);
+        // (u <= 1 + 2^-23, so bits(u) >> 17 <= 8128 stays inside the 8192-byte table)
+        t8 = ev.ld + 8u * lds_u8((ub >> 17) | ev.lut);
+        for (int s = 0; s < ev.refine; ++s) t8 = add8_if_le(t8, lds_f32(t8 + 8u), u);
+        t8 = min(t8, ev.ld + 8u * (uint32_t)(n - 2));
     }
     const float2 ld = lds_f32x2(t8);
     const float den = ld.y;

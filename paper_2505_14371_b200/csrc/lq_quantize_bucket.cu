@@ -122,7 +122,7 @@ __device__ __forceinline__ void bucket_norms8(const float4* ring_ptr, int q, int
 // replace the consumed ones (nullptr: nothing to fetch); `prev_rows` says which rows may be nonzero in the
 // previous message and lanes 0..7 of prev_norm8 hold that message's norms of rows 0..7.  Returns this lane's
 // statistic term.
-template <int B, bool kFast, bool kHist>
+template <int B, int kSearch, bool kHist>
 __device__ __forceinline__ double quantize_block(const PlanDev& p, const PhiloxConsts& pc, BucketCtx& c, QuantEnv ev,
                                                  int64_t blk, uint32_t prev_rows, const float* __restrict__ next,
                                                  uint32_t* __restrict__ out, const uint32_t (&pw)[B + 1],
@@ -170,7 +170,7 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const PhiloxC
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const bool counted = !kHist || blk * kBlockCoords + 128 * j + 4 * lane + e < c.size;
-                quantize_coord<B, kFast, kHist, true, true>(ev, vv[e], x[e], 4 * j + e, cw, pw, stat, nrow, pn, counted);
+                quantize_coord<B, kSearch, kHist, true, true>(ev, vv[e], x[e], 4 * j + e, cw, pw, stat, nrow, pn, counted);
             }
         } else {
             pack_zero_row<C>(cw, j, ev.ld);
@@ -189,7 +189,7 @@ __device__ __forceinline__ double quantize_block(const PlanDev& p, const PhiloxC
 }
 
 // A warp's share of a tile: blocks warp, warp + 8, ...
-template <int B, bool kFast, bool kHist>
+template <int B, int kSearch, bool kHist>
 __device__ __forceinline__ double quantize_tile(const PlanDev& p, const PhiloxConsts& pc, BucketCtx& c, const QuantEnv& ev,
                                                 const Tile& tile, uint32_t* __restrict__ out,
                                                 const uint32_t* __restrict__ prev)
@@ -227,7 +227,7 @@ __device__ __forceinline__ double quantize_tile(const PlanDev& p, const PhiloxCo
         const bool has_next = nb < tile.nblocks;
         const int64_t nblk = tile.block0 + nb;
         const float* next = (has_next && nblk < nfull) ? c.g + nblk * kBlockCoords + 4 * c.lane : nullptr;
-        stat += quantize_block<B, kFast, kHist>(p, pc, c, ev, blk, pmask, next, out, pw, prev_norm8);
+        stat += quantize_block<B, kSearch, kHist>(p, pc, c, ev, blk, pmask, next, out, pw, prev_norm8);
         primed = has_next;
         if (has_next && nblk >= nfull) issue_ragged_block(c, nblk);   // the layer's last, partial block
     }
@@ -251,10 +251,10 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_bucket_kernel(
     const int k = blockIdx.y + p.worker0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t kl = (int64_t)k * p.num_layers + layer;
-    const bool fast = st.fast[layer] != 0;
+    const int search = st.fast[layer];                      // 1: one lookup; 1 + R: byte table and up to R steps
 
     // the tables hold the plain levels (norm 1) and each row multiplies by its own norm
-    fill_tables(sm, st, layer, L.nlevels, fast, levels_cur, levels_prev, 1.0f, 1.0f, kHist);
+    fill_tables(sm, st, layer, L.nlevels, true, levels_cur, levels_prev, 1.0f, 1.0f, kHist);
     __syncthreads();
 
     BucketCtx c;
@@ -272,6 +272,7 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_bucket_kernel(
     QuantEnv ev;
     ev.lut = base + kSmLut; ev.ld = base + kSmLd; ev.tprev = base + kSmTprev;
     ev.r = 1.0f;
+    ev.refine = search - 1;
     ev.hist = reinterpret_cast<uint32_t*>(sm + kSmHist);
     if (step == LQ_STEP_AUTO) step = (uint32_t)p.scalars->t;      // the plan's own iteration counter (graph replays)
     const PhiloxConsts pc = philox_fold((uint32_t)layer, (uint32_t)k, step, p.seed_lo, p.seed_hi);
@@ -279,10 +280,10 @@ __global__ void __launch_bounds__(kQThreads, 3) quantize_pack_bucket_kernel(
     const uint32_t* prev = prev_packed ? prev_packed + (int64_t)k * p.packed_words + L.word_off : nullptr;
 
     double stat = 0.0;
-    switch (L.bits * 2 + (fast ? 1 : 0)) {
+    switch (L.bits * 2 + (search == 1 ? 1 : 0)) {
 #define LQ_CASE(BB)                                                                              \
-    case 2 * BB:     stat = quantize_tile<BB, false, kHist>(p, pc, c, ev, tile, out, prev); break;  \
-    case 2 * BB + 1: stat = quantize_tile<BB, true, kHist>(p, pc, c, ev, tile, out, prev); break;
+    case 2 * BB:     stat = quantize_tile<BB, 2, kHist>(p, pc, c, ev, tile, out, prev); break;  \
+    case 2 * BB + 1: stat = quantize_tile<BB, 1, kHist>(p, pc, c, ev, tile, out, prev); break;
         LQ_CASE(1) LQ_CASE(2) LQ_CASE(3) LQ_CASE(4) LQ_CASE(5) LQ_CASE(6) LQ_CASE(7) LQ_CASE(8)
 #undef LQ_CASE
         default: break;

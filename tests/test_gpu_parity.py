@@ -404,6 +404,43 @@ def test_qoda_step_more_than_32_workers(lqm, orc):
         assert _close(to_unpadded(plan, Y), model.Y, 1e-6) and _close(to_unpadded(plan, Xh), model.Xhalf, 1e-6)
 
 
+@pytest.mark.parametrize("bits", [5, 6, 8])
+def test_levels_crowded_into_one_search_bin(lqm, orc, bits):
+    """Level sets too dense for the one-lookup search (it takes at most one level per 1/32 of an octave): most
+    interior levels a few ulps apart just above 0.75, the rest spread out, with the max norm so that the normalised
+    values cover [0, 1] and many land between the crowded levels; then uniform 2^b levels, dense near 1 only.
+    Words, histogram and statistic against the oracle."""
+    n = 1 << bits
+    crowd = n - 2 - 6
+    lv = np.concatenate([[0.0], np.float32([1e-3, 0.02, 0.3, 0.74]),
+                         np.float32(0.75) + np.arange(1, crowd + 1, dtype=np.float32) * np.float32(2.0 ** -22),
+                         np.float32([0.9, 0.99]), [1.0]]).astype(np.float32)
+    assert lv.size == n and np.all(np.diff(lv) > 0)
+    sizes = [5000, 70001]
+    plan = lqm.Plan(sizes, bits, 0, 2, SEED + bits)
+    plan.lq_set_levels(0, lv)                                  # layer 1 keeps the uniform levels
+    g = torch.Generator(device="cuda").manual_seed(bits)
+    grads = torch.rand((2, plan.padded_elems), generator=g, device="cuda") * 2 - 1
+    near = np.float32(0.75) + np.float32(2.0 ** -22) * torch.rand(2000, generator=g, device="cuda") * crowd
+    grads[:, 100:2100] = near                                  # values between the crowded levels
+    grads[:, 0] = 1.0                                          # the max norm is exactly 1
+    packed = plan.empty_packed(); norms = plan.empty_norms(); hist = plan.zero_hist()
+    plan.lq_quantize_pack(grads, 3, packed, norms, hist=hist)
+    model = oracle_model(orc, plan)
+    model.levels[0] = lv
+    ref = model.quantize(to_unpadded(plan, grads), 3, want_hist=True)
+    assert np.array_equal(norms.cpu().numpy()[:, :plan.num_layers], ref["norms"])
+    assert compare_messages(orc, plan, packed, ref) == (0, 0)
+    assert np.array_equal(hist.cpu().numpy().view(np.uint32), ref["hist"])
+    packed2 = plan.empty_packed(); norms2 = plan.empty_norms()
+    plan.lq_quantize_pack(grads, 4, packed2, norms2, prev_packed=packed, prev_norms=norms)
+    model.prev_decoded = ref["decoded"]
+    ref2 = model.quantize(to_unpadded(plan, grads), 4)
+    assert compare_messages(orc, plan, packed2, ref2) == (0, 0)
+    sq, _ = plan.lq_get_statistics()
+    assert _close(sq.numpy(), ref2["sq_diff"], 1e-12)
+
+
 def test_argument_errors(lqm):
     with pytest.raises(lqm.LqError):
         lqm.Plan([10], 9, 2, 1, 0)
