@@ -15,7 +15,7 @@
 // instruction issue (about 42 instructions per coordinate: 10 Philox, 7 the statistic), not by DRAM.
 //
 // The level search and the tables are described in lq_quantize.cuh.  Layers whose levels are denser than the
-// search table's bins fall back to a binary search.
+// search table's bins take a byte table over finer bins and step up from its entry (build_search_kernel).
 //
 // The norm pass, which reads the same values just before, leaves one bit per row of 128 values
 // that says whether the row holds anything but zeros.  An all-zero row (untouched embedding rows)
