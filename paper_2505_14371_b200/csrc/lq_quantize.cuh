@@ -240,8 +240,8 @@ __device__ __forceinline__ void quantize_coord(const QuantEnv& ev, float v, uint
         const uint32_t e = lds_u32(((ub >> 17) & 0x1FFCu) | ev.lut);
         t8 = add8_if_gt_u32((e & 0x7F8u) | ev.ld, ub << 13, e);
     } else {
-        // (u <= 1 + 2^-23, so bits(u) >> 17 <= 8128 stays inside the 8192-byte table)
-        t8 = ev.ld + 8u * lds_u8((ub >> 17) | ev.lut);
+        // (u <= 1 + 2^-23 gives bits(u) >> 17 <= 8128; the mask keeps the pattern of a NaN inside the table too)
+        t8 = ev.ld + 8u * lds_u8(((ub >> 17) & 0x1FFFu) | ev.lut);
         for (int s = 0; s < ev.refine; ++s) t8 = add8_if_le(t8, lds_f32(t8 + 8u), u);
         t8 = min(t8, ev.ld + 8u * (uint32_t)(n - 2));
     }
