@@ -130,30 +130,31 @@ __device__ __forceinline__ uint32_t lane_bits(const uint32_t* code, const uint32
     return bits;
 }
 
-// Writes a lane's coordinates into the block's buffer from bit `pos` on.  The lane's bits gather in {lo, hi} and leave
-// one whole word at a time: the first and the last word it touches may be shared with its neighbours (atomic OR into
-// the zeroed buffer), the words between them are its own (plain stores).
+// Writes a lane's coordinates into the block's buffer from bit `pos` on.  The lane's bits gather in a 64-bit word and
+// leave 32 at a time: the first and the last word it touches may be shared with its neighbours (atomic OR into the
+// zeroed buffer), the words between them are its own (plain stores).  Whole blocks are taken two coordinates at a
+// time: with fewer than 32 bits waiting, two coordinates (at most 26 bits) still fit.
 template <int C, bool kFull>
 __device__ __forceinline__ void lane_emit(const uint32_t* code, const uint32_t (&w)[C + 1], int64_t blk, int lane,
                                           int64_t size, uint32_t pos, uint32_t* buf)
 {
-    uint32_t lo = 0, hi = 0, f = pos & 31u;
+    uint64_t acc = 0;
+    uint32_t f = pos & 31u;
     uint32_t* dst = buf + (pos >> 5);
     bool first = true;
 #pragma unroll
     for (int pp = 0; pp < 32; ++pp) {
         if (!kFull && !real_coord(blk, lane, pp, size)) continue;
-        const uint32_t e = code[symbol_at<C>(w, pp)], val = e & 0xffffu;
-        lo |= val << f;
-        hi |= __funnelshift_l(val, 0u, f);                    // the bits of val << f above bit 31
+        const uint32_t e = code[symbol_at<C>(w, pp)];
+        acc |= (uint64_t)(e & 0xffffu) << f;
         f += e >> 16;
-        if (f >= 32u) {
-            if (first) atomicOr(dst, lo); else *dst = lo;
+        if ((kFull ? (pp & 1) == 1 : true) && f >= 32u) {
+            if (first) atomicOr(dst, (uint32_t)acc); else *dst = (uint32_t)acc;
             first = false;
-            ++dst; lo = hi; hi = 0u; f -= 32u;
+            ++dst; acc >>= 32; f -= 32u;
         }
     }
-    if (f) atomicOr(dst, lo);
+    if (f) atomicOr(dst, (uint32_t)acc);
 }
 
 constexpr int kCodeBufWords = kBlockCoords * (kCodeMaxLen + 1) / 32;      // longest block: every coordinate 13 bits
